@@ -1,0 +1,237 @@
+/*
+ * moin.h - C ABI of the MoIN serving hot path for NVIDIA B200 (sm_100a).
+ *
+ * MoIN ("Mixture of Introvert Experts") routes every request to ONE expert - a LoRA adapter
+ * on a frozen dense base model - and runs the whole forward pass with that adapter.  This
+ * library is the data-parallel hot path of serving such a model on one GPU:
+ *
+ *   moin_route            query embedding -> nearest topic embedding -> expert id
+ *   moin_plan_build       group the tokens of a batch by expert (once per batch)
+ *   moin_lora_linear      y = x W^T + s (x A_e^T) B_e^T with the expert e differing per token
+ *   moin_decoder_forward  Llama-architecture decoder whose seven per-block projections are
+ *                         that layer
+ *
+ * General conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller unless the comment says
+ *     "host".  The library borrows it for the duration of the call's work on `stream`; it
+ *     never frees it and never allocates device memory itself (scratch comes in through the
+ *     `workspace` arguments, sized by the *_workspace_bytes queries).
+ *   - Descriptor structs (moin_router, moin_pool, moin_plan, moin_model) are plain host
+ *     structs filled by the caller; arrays of pointers inside moin_model are HOST arrays of
+ *     device pointers.
+ *   - Matrices are row-major, bf16 (IEEE bfloat16 bit patterns) unless stated; device
+ *     pointers to bf16/fp32 tensors must be 16-byte aligned (MOIN_ERR_MISALIGNED otherwise).
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the legacy
+ *     default stream) except where a comment says the call synchronises.  Errors that the
+ *     host can detect are returned at once and nothing is launched.  Conditions only the
+ *     device can see (an expert id outside [0, E), a bounded wait that ran out) never trap or
+ *     hang: an out-of-range id means "no adapter" and is counted, a wait that runs out sets a
+ *     flag, the kernel returns; both are read back with moin_device_status.
+ *   - Results are deterministic: identical inputs give bit-identical outputs run to run.
+ *   - Arithmetic: bf16 operands, fp32 accumulation, one rounding to bf16 at the output.
+ */
+#ifndef MOIN_H_
+#define MOIN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t moin_status;
+typedef void* moin_stream; /* cudaStream_t */
+
+enum {
+  MOIN_OK = 0,
+  MOIN_ERR_INVALID_ARG = -1,      /* null pointer, negative size */
+  MOIN_ERR_BAD_SHAPE = -2,        /* a dimension violates the documented divisibility rules */
+  MOIN_ERR_MISALIGNED = -3,       /* a tensor pointer is not 16-byte aligned */
+  MOIN_ERR_WORKSPACE = -4,        /* workspace too small or null */
+  MOIN_ERR_UNSUPPORTED_RANK = -5, /* LoRA rank not a multiple of 8 in 8..64 */
+  MOIN_ERR_CUDA = -6,             /* a CUDA runtime/driver call failed (see moin_last_cuda_error) */
+  MOIN_ERR_TIMEOUT = -7,          /* a device-side bounded wait ran out (reported by moin_device_status) */
+  MOIN_ERR_NO_DEVICE = -8         /* no sm_100 device is current */
+};
+
+/* Human-readable name of a status code (static string). */
+const char* moin_status_string(moin_status s);
+/* Library version, major*10000 + minor*100 + patch. */
+int32_t moin_version(void);
+/* cudaError_t value of the last failing CUDA call seen by this library on this thread (0 = none). */
+int32_t moin_last_cuda_error(void);
+
+/* Device-side condition counters, accumulated since the last moin_device_status_reset. */
+typedef struct {
+  int32_t timeout_flag;       /* != 0: some bounded wait ran out; results of that call are undefined */
+  int32_t timeout_site;       /* small integer naming the wait that gave up (diagnostic) */
+  int32_t invalid_expert_ids; /* token expert ids outside [-1, E) seen by moin_plan_build (treated as -1) */
+  int32_t reserved[5];
+} moin_device_status_t;
+/* Copies the counters to *out (host).  SYNCHRONISES `stream`. */
+moin_status moin_device_status(moin_device_status_t* out, moin_stream stream);
+moin_status moin_device_status_reset(moin_stream stream);
+
+/* Testing/tuning knobs (host-side path selection only; every path computes the same function).
+ *   MOIN_OPT_GEMM_IMPL: 0 = automatic, 1 = force the warp-MMA kernels, 2 = force the tcgen05 kernels
+ *                       (calls whose shapes the forced kernel cannot take fail with MOIN_ERR_BAD_SHAPE). */
+enum { MOIN_OPT_GEMM_IMPL = 1 };
+moin_status moin_set_option(int32_t key, int32_t value);
+
+/* ---------------------------------------------------------------------------------------
+ * Router.  Paper Sec. 3.3 (model inference): the query is embedded and a nearest-neighbour
+ * search over the topic embeddings picks the expert; the metric used here is the cosine
+ * similarity, lowest index on exact ties.
+ *
+ *   id_i = argmax_k <q_i, c_k> / (|q_i| |c_k|)
+ *
+ * |q_i| is a positive per-query constant and is not needed for the argmax; |c_k| is, because
+ * bf16-rounded "unit" vectors are not unit.  A zero-norm centroid has similarity -inf.
+ * Similarities are accumulated in fp32 and compared in fp32.
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  const void* centroids;             /* [K, D] bf16 topic embeddings */
+  const float* inv_norm;             /* [K] fp32, 1/|c_k| (0 for a zero-norm row); see moin_router_prepare */
+  const int32_t* centroid_to_expert; /* [K] int32 or NULL: expert id of each topic, -1 = topic has no adapter
+                                        (paper Sec. 4: some clusters were not retained) */
+  int32_t K;                         /* number of topic embeddings, >= 1 */
+  int32_t D;                         /* embedding dimension, multiple of 8, 8 <= D <= 8192 */
+} moin_router;
+
+/* Fills inv_norm[K] (fp32, device) from centroids[K, D].  Once per centroid table. */
+moin_status moin_router_prepare(const void* centroids, int32_t K, int32_t D, float* inv_norm, moin_stream stream);
+
+size_t moin_route_workspace_bytes(int32_t Q, int32_t K, int32_t D);
+/* queries [Q, D] bf16 -> out_expert[Q] (int32: centroid_to_expert[id] if the map is given, else id),
+ * out_centroid[Q] (nullable, int32 id), out_best_sim[Q] (nullable, fp32 cosine of the winner).
+ * Q == 0 is a no-op.  Workspace contents are scratch. */
+moin_status moin_route(const moin_router* router, const void* queries, int32_t Q, int32_t* out_expert,
+                       int32_t* out_centroid, float* out_best_sim, void* workspace, size_t workspace_bytes,
+                       moin_stream stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Adapter pool of ONE projection.  Paper Sec. 3.2: W_a in R^{r x d}, W_b in R^{k x r} per
+ * expert and linear layer; Sec. 1: the adapters in use are kept in GPU memory.  The pool
+ * stores the paper's matrices as written, stacked over slots:
+ *   A[n_slots, r, d_in] = W_a,  B[n_slots, d_out, r] = W_b,
+ * and slot_of_expert[E] maps an expert id to its slot, -1 = the expert has no adapter
+ * (paper Sec. 4: then the base model alone is used).
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  const void* A;
+  const void* B;
+  const int32_t* slot_of_expert; /* [E] int32, values in [-1, n_slots) */
+  int32_t E;
+  int32_t n_slots;
+  int32_t r;     /* LoRA rank: multiple of 8, 8..64 */
+  int32_t d_in;  /* multiple of 64 */
+  int32_t d_out; /* multiple of 8 */
+} moin_pool;
+
+/* ---------------------------------------------------------------------------------------
+ * Batch plan = the grouping of a batch's tokens by expert.  Paper Sec. 1 names the need
+ * (many adapters in one batch) and Sec. 3.3 fixes that the expert is per request, so the
+ * plan is built once per batch and reused by every projection of every block.
+ *
+ * The plan lives in a caller-provided device buffer of moin_plan_bytes(T, E) bytes and holds
+ *   - a stable permutation of token indices ordered by expert id, with one segment
+ *     (expert, start, length) per distinct expert - used when segments are short (decode);
+ *   - the list of row tiles: maximal runs of consecutive tokens with one expert, cut into
+ *     pieces of at most 128 rows - used when runs are long (prefill).
+ * Token expert ids: -1 = no expert (base model only); ids outside [-1, E) are treated as -1
+ * and counted in moin_device_status.
+ * ------------------------------------------------------------------------------------- */
+enum {
+  MOIN_PLAN_AUTO = 0,     /* choose from the built plan; moin_plan_build then SYNCHRONISES the stream */
+  MOIN_PLAN_SEGMENTS = 1, /* short segments: stream each distinct adapter once over sorted tokens */
+  MOIN_PLAN_TILES = 2     /* long runs: adapter folded into the tensor-core GEMM tile by tile */
+};
+typedef struct {
+  void* buffer;        /* device, moin_plan_bytes(T, E) bytes, 16-byte aligned */
+  size_t buffer_bytes;
+  int32_t T;           /* tokens in the batch */
+  int32_t E;           /* expert ids are in [0, E) */
+  int32_t mode;        /* in: MOIN_PLAN_AUTO/SEGMENTS/TILES; out (AUTO only): the mode chosen */
+  /* host-visible summary, filled only by an AUTO build (which synchronises): */
+  int32_t n_segments, n_tiles, n_lora_tokens, max_segment;
+} moin_plan;
+
+size_t moin_plan_bytes(int32_t T, int32_t E);
+/* token_expert [T] int32 (device).  Fills plan->buffer.  T == 0 is a no-op. */
+moin_status moin_plan_build(const int32_t* token_expert, moin_plan* plan, moin_stream stream);
+
+/* Copies the plan's arrays to host memory for inspection (tests).  Any pointer may be NULL.
+ * perm[T]; seg_expert[S], seg_start[S+1] with S = *n_segments; tile_row0/rows/expert[n_tiles].
+ * Output arrays must have room for T + 1 entries.  SYNCHRONISES `stream`. */
+moin_status moin_plan_read(const moin_plan* plan, int32_t* n_segments, int32_t* n_tiles, int32_t* perm,
+                           int32_t* seg_expert, int32_t* seg_start, int32_t* tile_row0, int32_t* tile_rows,
+                           int32_t* tile_expert, moin_stream stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Routed LoRA linear layer.  Paper Sec. 3.2: y = W x + W_b (W_a x), W in R^{k x d}; the
+ * expert is the request's (Sec. 3.3); no adapter => W x only (Sec. 4).  With a scale s on
+ * the low-rank term (s = 1 is the paper's formula):
+ *
+ *   y[t, :] = x[t, :] W^T + s * (x[t, :] A_e^T) B_e^T,   e = expert of token t
+ *
+ *   x [T, d_in] bf16, W [d_out, d_in] bf16, y [T, d_out] bf16 (must not alias x).
+ *   pool == NULL (or plan == NULL): base layer only; then T, d_in, d_out come from base_T,
+ *   base_d_in, base_d_out (ignored otherwise: plan->T and the pool give them).
+ *   fp32 accumulation of the base and the low-rank term, added in fp32, rounded once to bf16.
+ *   T == 0 is a no-op.  Workspace contents are scratch.
+ * ------------------------------------------------------------------------------------- */
+size_t moin_lora_linear_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, int32_t r);
+moin_status moin_lora_linear(const moin_plan* plan, const void* x, const void* W, const moin_pool* pool,
+                             float scale, int32_t base_T, int32_t base_d_in, int32_t base_d_out, void* y,
+                             void* workspace, size_t workspace_bytes, moin_stream stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Decoder forward.  Paper Sec. 4: the base model is TinyLlama-1.1B (Llama-2 architecture);
+ * Sec. 3.2: an adapter on each linear layer; Sec. 3.3: the request's expert for the whole
+ * forward pass.  Conventions (the paper fixes none): pre-norm blocks; RMSNorm with gain;
+ * rotary embedding pairing (i, i + head_dim/2), angle pos * rope_base^(-2i/head_dim),
+ * positions restart at 0 per request; causal softmax attention within each request, scale
+ * 1/sqrt(head_dim); query head h reads kv head h / (n_heads / n_kv_heads);
+ * down(silu(gate(v)) * up(v)); no biases; untied lm_head; no adapter on embedding / lm_head.
+ * Storage: residual stream fp32; norm outputs, projection outputs, rotated q/k, attention
+ * output, SwiGLU output and logits bf16.  head_dim must be 64.
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t n_layers, hidden, n_heads, n_kv_heads, head_dim, ffn, vocab;
+  float rms_eps, rope_base, lora_scale;
+  const void* embed;             /* [vocab, hidden] bf16 */
+  const void* lm_head;           /* [vocab, hidden] bf16 */
+  const void* final_norm;        /* [hidden] bf16 gain */
+  const void* const* attn_norm;  /* host array [n_layers] of device [hidden] bf16 */
+  const void* const* mlp_norm;   /* host array [n_layers] of device [hidden] bf16 */
+  const void* const* W;          /* host array [n_layers*7] of device [d_out, d_in] bf16; order q,k,v,o,gate,up,down */
+  const moin_pool* pools;        /* host array [n_layers*7] or NULL (base model) */
+  int32_t E;                     /* expert ids in [0, E) */
+} moin_model;
+
+/* Optional taps for block-by-block checks.  hidden_in (nullable, [T, hidden] fp32): start from this
+ * residual stream instead of the embedding lookup; blocks [layer_begin, layer_end) are applied;
+ * hidden_out (nullable, [T, hidden] fp32) receives the residual stream after them. */
+typedef struct {
+  const float* hidden_in;
+  float* hidden_out;
+  int32_t layer_begin, layer_end;
+} moin_decoder_taps;
+
+enum { MOIN_LOGITS_ALL = 0, MOIN_LOGITS_LAST = 1, MOIN_LOGITS_NONE = 2 };
+
+size_t moin_decoder_workspace_bytes(const moin_model* model, int32_t R, int32_t T);
+/* tokens [T] int32 packed request-major; cu_seqlens [R+1] int32 (cu[0] = 0, cu[R] = T);
+ * req_expert [R] int32 (-1 = base only).  max_seqlen: host upper bound on a request's length.
+ * logits: [T, vocab] bf16 (MOIN_LOGITS_ALL - what a perplexity evaluation needs) or [R, vocab]
+ * (MOIN_LOGITS_LAST: last token of each request) or unused (MOIN_LOGITS_NONE). */
+moin_status moin_decoder_forward(const moin_model* model, const int32_t* tokens, const int32_t* cu_seqlens,
+                                 const int32_t* req_expert, int32_t R, int32_t T, int32_t max_seqlen,
+                                 void* logits, int32_t logits_mode, const moin_decoder_taps* taps,
+                                 void* workspace, size_t workspace_bytes, moin_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOIN_H_ */

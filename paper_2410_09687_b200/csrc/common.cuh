@@ -1,0 +1,111 @@
+// Shared device/host helpers of the MoIN CUDA library (sm_100a only).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <limits.h>
+#include <stdint.h>
+
+#include "../../include/moin.h"
+
+namespace moin {
+
+// ----------------------------------------------------------------------------------------
+// Device status block (one per process; its device address is passed to kernels).
+// ----------------------------------------------------------------------------------------
+struct DeviceStatus {
+  int timeout_flag;
+  int timeout_site;
+  int invalid_expert_ids;
+  int reserved[5];
+};
+
+// Plan buffer layout (int32 words).  Header first, then the arrays.
+constexpr int kPlanHeaderWords = 16;
+enum PlanHeader { PH_NSEG = 0, PH_NTILES = 1, PH_NLORA = 2, PH_MAXSEG = 3, PH_T = 4, PH_E = 5 };
+constexpr int kPlanChunk = 256;   // tokens per histogram chunk
+constexpr int kTileRows = 128;    // rows per GEMM tile
+
+struct PlanView {   // pointers into the plan buffer
+  int* header;
+  int* perm;         // [T]   token indices ordered by (expert, token)
+  int* seg_expert;   // [Smax]
+  int* seg_start;    // [Smax + 1]
+  int* tile_row0;    // [T + 1]
+  int* tile_rows;    // [T]
+  int* tile_expert;  // [T]
+  int* rank;         // [T]   scratch
+  int* key;          // [T]   scratch
+  int* keybase;      // [E+1] scratch
+  int* hist;         // [n_chunks * (E+1)] scratch
+  int T, E, Smax, n_chunks;
+};
+
+__host__ __device__ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline PlanView plan_view(void* buffer, int T, int E, size_t* total_words = nullptr) {
+  PlanView v;
+  v.T = T; v.E = E;
+  v.Smax = T < E ? T : E;
+  v.n_chunks = (T + kPlanChunk - 1) / kPlanChunk;
+  int* base = reinterpret_cast<int*>(buffer);
+  size_t off = 0;
+  auto take = [&](size_t n) { size_t o = off; off += align_up(n, 4); return base ? base + o : nullptr; };
+  v.header = take(kPlanHeaderWords);
+  v.perm = take(T);
+  v.seg_expert = take(v.Smax + 1);
+  v.seg_start = take(v.Smax + 2);
+  v.tile_row0 = take(T + 1);
+  v.tile_rows = take(T + 1);
+  v.tile_expert = take(T + 1);
+  v.rank = take(T);
+  v.key = take(T);
+  v.keybase = take(E + 2);
+  v.hist = take((size_t)v.n_chunks * (size_t)(E + 1));
+  if (total_words) *total_words = off;
+  return v;
+}
+inline size_t plan_bytes(int T, int E) {
+  size_t words = 0;
+  plan_view(nullptr, T, E, &words);
+  return words * sizeof(int);
+}
+
+// ----------------------------------------------------------------------------------------
+// Small device utilities
+// ----------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Streaming 16-byte load that does not allocate in L1 (adapter weights are read once).
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint4 ldg_cached(const void* p) {
+  return __ldg(reinterpret_cast<const uint4*>(p));
+}
+
+// mma.sync m16n8k16, bf16 x bf16 -> fp32 (warp-level tensor-core path for the skinny LoRA products)
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Launchers implemented in the .cu files (host side).
+cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, DeviceStatus* status, cudaStream_t stream);
+
+}  // namespace moin

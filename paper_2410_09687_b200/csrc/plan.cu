@@ -1,0 +1,191 @@
+// Batch plan: grouping of tokens by expert id (integer work only).
+//
+// Three small launches:
+//   plan_rank_kernel    per 256-token chunk: sanitise ids, stable in-chunk rank, per-chunk histogram
+//   plan_scan_kernel    one CTA: prefix over chunks and over expert ids -> segment list; run tiles
+//   plan_scatter_kernel per chunk: position = expert base + chunk prefix + in-chunk rank -> perm
+// The result is a stable counting sort (token order is kept inside every expert segment), so
+// the plan is deterministic.
+#include "common.cuh"
+
+namespace moin {
+
+__global__ void __launch_bounds__(kPlanChunk) plan_rank_kernel(const int* __restrict__ token_expert, int T, int E,
+                                                               int* __restrict__ key, int* __restrict__ rank,
+                                                               int* __restrict__ hist, DeviceStatus* status) {
+  __shared__ int skey[kPlanChunk];
+  const int tid = threadIdx.x;
+  const int t = blockIdx.x * kPlanChunk + tid;
+  int k = -2;  // padding lanes never match
+  if (t < T) {
+    int e = token_expert[t];
+    if (e >= 0 && e < E) {
+      k = e;
+    } else {
+      k = E;  // "no adapter" bucket
+      if (e != -1) atomicAdd(&status->invalid_expert_ids, 1);
+    }
+  }
+  skey[tid] = k;
+  __syncthreads();
+  if (t >= T) return;
+  int before = 0, after = 0;
+  for (int i = 0; i < kPlanChunk; ++i) {
+    int same = (skey[i] == k);
+    before += same & (i < tid);
+    after += same & (i > tid);
+  }
+  key[t] = k;
+  rank[t] = before;
+  if (after == 0) hist[(size_t)blockIdx.x * (size_t)(E + 1) + k] = before + 1;
+}
+
+// Block-wide scans for 1024 threads.  `smem` must hold 33 ints.
+__device__ __forceinline__ int block_excl_sum_1024(int v, int* smem, int* total) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int n = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += n;
+  }
+  __syncthreads();  // protect smem reuse between calls
+  if (lane == 31) smem[w] = inc;
+  __syncthreads();
+  if (w == 0) {
+    int s = smem[lane];
+    int si = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int n = __shfl_up_sync(0xffffffffu, si, o);
+      if (lane >= o) si += n;
+    }
+    smem[lane] = si - s;  // exclusive prefix of warp totals
+    if (lane == 31) smem[32] = si;
+  }
+  __syncthreads();
+  *total = smem[32];
+  return smem[w] + inc - v;
+}
+__device__ __forceinline__ int block_incl_max_1024(int v, int* smem) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int n = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc = max(inc, n);
+  }
+  __syncthreads();
+  if (lane == 31) smem[w] = inc;
+  __syncthreads();
+  if (w == 0) {
+    int s = smem[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int n = __shfl_up_sync(0xffffffffu, s, o);
+      if (lane >= o) s = max(s, n);
+    }
+    smem[lane] = s;  // inclusive max over warps 0..lane
+  }
+  __syncthreads();
+  int prev = (w > 0) ? smem[w - 1] : INT_MIN;
+  return max(inc, prev);
+}
+
+__global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v) {
+  __shared__ int smem[33];
+  __shared__ int s_carry[2];
+  const int tid = threadIdx.x;
+  const int T = v.T, E = v.E, nc = v.n_chunks;
+  const size_t pitch = (size_t)(E + 1);
+
+  // 1. per expert id: prefix over chunks (in place) and total
+  for (int k = tid; k <= E; k += 1024) {
+    int run = 0;
+    for (int c = 0; c < nc; ++c) {
+      int* p = v.hist + (size_t)c * pitch + k;
+      int n = *p;
+      *p = run;
+      run += n;
+    }
+    v.keybase[k] = run;
+  }
+  __syncthreads();
+
+  // 2. prefix over expert ids -> segment list (ascending expert id), "no adapter" bucket last
+  int carry_tok = 0, carry_seg = 0, max_seg = 0;
+  for (int k0 = 0; k0 < E; k0 += 1024) {
+    int k = k0 + tid;
+    int n = (k < E) ? v.keybase[k] : 0;
+    int tot_tok, tot_seg;
+    int ex_tok = block_excl_sum_1024(n, smem, &tot_tok);
+    int ex_seg = block_excl_sum_1024(n > 0 ? 1 : 0, smem, &tot_seg);
+    if (k < E) {
+      v.keybase[k] = carry_tok + ex_tok;
+      if (n > 0) {
+        v.seg_expert[carry_seg + ex_seg] = k;
+        v.seg_start[carry_seg + ex_seg] = carry_tok + ex_tok;
+      }
+    }
+    max_seg = max(max_seg, n);
+    carry_tok += tot_tok;
+    carry_seg += tot_seg;
+  }
+  max_seg = block_incl_max_1024(max_seg, smem);
+  if (tid == 1023) {
+    v.seg_start[carry_seg] = carry_tok;
+    v.keybase[E] = carry_tok;
+    v.header[PH_NSEG] = carry_seg;
+    v.header[PH_NLORA] = carry_tok;
+    v.header[PH_MAXSEG] = max_seg;
+    v.header[PH_T] = T;
+    v.header[PH_E] = E;
+  }
+
+  // 3. row tiles: maximal runs of equal expert id in token order, cut every kTileRows rows
+  int carry_start = 0, carry_tiles = 0;
+  for (int t0 = 0; t0 < T; t0 += 1024) {
+    int t = t0 + tid;
+    int k = (t < T) ? v.key[t] : -3;
+    int is_start = (t < T) && (t == 0 || v.key[t - 1] != k);
+    int rs = block_incl_max_1024(is_start ? t : -1, smem);
+    rs = max(rs, carry_start);
+    int flag = (t < T) && (((t - rs) % kTileRows) == 0);
+    int tot;
+    int idx = carry_tiles + block_excl_sum_1024(flag, smem, &tot);
+    if (flag) {
+      v.tile_row0[idx] = t;
+      v.tile_expert[idx] = (k == E) ? -1 : k;
+    }
+    if (tid == 1023) s_carry[0] = rs;
+    __syncthreads();
+    carry_start = s_carry[0];
+    carry_tiles += tot;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    v.tile_row0[carry_tiles] = T;
+    v.header[PH_NTILES] = carry_tiles;
+  }
+  __syncthreads();
+  for (int i = tid; i < carry_tiles; i += 1024) v.tile_rows[i] = v.tile_row0[i + 1] - v.tile_row0[i];
+}
+
+__global__ void __launch_bounds__(kPlanChunk) plan_scatter_kernel(PlanView v) {
+  const int t = blockIdx.x * kPlanChunk + threadIdx.x;
+  if (t >= v.T) return;
+  const int k = v.key[t];
+  const int pos = v.keybase[k] + v.hist[(size_t)blockIdx.x * (size_t)(v.E + 1) + k] + v.rank[t];
+  v.perm[pos] = t;
+}
+
+cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, DeviceStatus* status, cudaStream_t stream) {
+  cudaError_t e = cudaMemsetAsync(v.hist, 0, sizeof(int) * (size_t)v.n_chunks * (size_t)(v.E + 1), stream);
+  if (e != cudaSuccess) return e;
+  plan_rank_kernel<<<v.n_chunks, kPlanChunk, 0, stream>>>(token_expert, v.T, v.E, v.key, v.rank, v.hist, status);
+  plan_scan_kernel<<<1, 1024, 0, stream>>>(v);
+  plan_scatter_kernel<<<v.n_chunks, kPlanChunk, 0, stream>>>(v);
+  return cudaGetLastError();
+}
+
+}  // namespace moin
