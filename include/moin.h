@@ -79,6 +79,25 @@ moin_status moin_device_status_reset(moin_stream stream);
 enum { MOIN_OPT_GEMM_IMPL = 1 };
 moin_status moin_set_option(int32_t key, int32_t value);
 
+/* Per-kernel timing for benchmarks (no counterpart in the paper).  While enabled, every kernel group the
+ * library launches is bracketed by a pair of CUDA events on the call's stream (this adds launch gaps:
+ * never leave it on for a throughput measurement).  moin_profile_enable(capacity > 0) pre-creates the
+ * events; capacity == 0 disables and frees them.  moin_profile_read SYNCHRONISES the device, writes up to
+ * `capacity` records in launch order, sets *n to the number recorded since the last read, and clears them. */
+typedef struct {
+  int32_t kernel;   /* MOIN_K_* */
+  int32_t launches; /* kernel launches inside the bracket */
+  float ms;         /* device time between the two events */
+} moin_profile_record;
+enum {
+  MOIN_K_ROUTE_SIMPLE = 0, MOIN_K_ROUTE_TC = 1, MOIN_K_ROUTE_FINISH = 2, MOIN_K_PLAN = 3, MOIN_K_GEMM_WARP = 4,
+  MOIN_K_GEMM_TC = 5, MOIN_K_SHRINK_STREAM = 6, MOIN_K_EXPAND_STREAM = 7, MOIN_K_SHRINK_TC = 8,
+  MOIN_K_FUSED_TC = 9, MOIN_K_GLUE = 10, MOIN_K_ATTENTION = 11, MOIN_K_COUNT = 12
+};
+moin_status moin_profile_enable(int32_t capacity);
+moin_status moin_profile_read(moin_profile_record* out, int32_t capacity, int32_t* n);
+const char* moin_kernel_name(int32_t kernel);
+
 /* ---------------------------------------------------------------------------------------
  * Router.  Paper Sec. 3.3 (model inference): the query is embedded and a nearest-neighbour
  * search over the topic embeddings picks the expert; the metric used here is the cosine

@@ -1,0 +1,371 @@
+// C ABI entry points: argument validation, workspace carving, kernel launches.
+#include <string.h>
+
+#include "common.cuh"
+#include "tc_gemm.cuh"
+
+namespace moin {
+
+__device__ DeviceStatus g_device_status;
+
+static thread_local int t_last_cuda_error = 0;
+static HostState g_state;
+
+moin_status record_cuda(cudaError_t e) {
+  if (e == cudaSuccess) return MOIN_OK;
+  t_last_cuda_error = (int)e;
+  return MOIN_ERR_CUDA;
+}
+
+moin_status host_state(HostState** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) { record_cuda(e); return MOIN_ERR_NO_DEVICE; }
+  if (g_state.device != dev) {
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, dev);
+    if (e != cudaSuccess) { record_cuda(e); return MOIN_ERR_NO_DEVICE; }
+    if (prop.major != 10) return MOIN_ERR_NO_DEVICE;  // built for sm_100a only
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_device_status);
+    if (e != cudaSuccess) return record_cuda(e);
+    g_state.status = reinterpret_cast<DeviceStatus*>(p);
+    g_state.n_sms = prop.multiProcessorCount;
+    g_state.device = dev;
+  }
+  *out = &g_state;
+  return MOIN_OK;
+}
+
+// ---- profiling (per-kernel CUDA events; off by default)
+struct ProfState {
+  int capacity = 0, count = 0;
+  cudaEvent_t* start = nullptr;
+  cudaEvent_t* stop = nullptr;
+  int* kernel = nullptr;
+  int* launches = nullptr;
+};
+static ProfState g_prof;
+
+ProfScope::ProfScope(int kernel, int launches, cudaStream_t s) : slot(-1), stream(s) {
+  if (g_prof.capacity > 0 && g_prof.count < g_prof.capacity) {
+    slot = g_prof.count++;
+    g_prof.kernel[slot] = kernel;
+    g_prof.launches[slot] = launches;
+    cudaEventRecord(g_prof.start[slot], stream);
+  }
+}
+ProfScope::~ProfScope() {
+  if (slot >= 0) cudaEventRecord(g_prof.stop[slot], stream);
+}
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace moin
+
+using namespace moin;
+
+extern "C" {
+
+const char* moin_status_string(moin_status s) {
+  switch (s) {
+    case MOIN_OK: return "MOIN_OK";
+    case MOIN_ERR_INVALID_ARG: return "MOIN_ERR_INVALID_ARG";
+    case MOIN_ERR_BAD_SHAPE: return "MOIN_ERR_BAD_SHAPE";
+    case MOIN_ERR_MISALIGNED: return "MOIN_ERR_MISALIGNED";
+    case MOIN_ERR_WORKSPACE: return "MOIN_ERR_WORKSPACE";
+    case MOIN_ERR_UNSUPPORTED_RANK: return "MOIN_ERR_UNSUPPORTED_RANK";
+    case MOIN_ERR_CUDA: return "MOIN_ERR_CUDA";
+    case MOIN_ERR_TIMEOUT: return "MOIN_ERR_TIMEOUT";
+    case MOIN_ERR_NO_DEVICE: return "MOIN_ERR_NO_DEVICE";
+    default: return "MOIN_ERR_UNKNOWN";
+  }
+}
+
+int32_t moin_version(void) { return 100; }
+int32_t moin_last_cuda_error(void) { return t_last_cuda_error; }
+
+moin_status moin_set_option(int32_t key, int32_t value) {
+  if (key == MOIN_OPT_GEMM_IMPL && value >= 0 && value <= 2) {
+    g_state.gemm_impl = value;
+    return MOIN_OK;
+  }
+  return MOIN_ERR_INVALID_ARG;
+}
+
+moin_status moin_device_status(moin_device_status_t* out, moin_stream stream) {
+  if (!out) return MOIN_ERR_INVALID_ARG;
+  HostState* hs;
+  moin_status st = host_state(&hs);
+  if (st) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  static_assert(sizeof(moin_device_status_t) == sizeof(DeviceStatus), "status layout");
+  cudaError_t e = cudaMemcpyAsync(out, hs->status, sizeof(DeviceStatus), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  return record_cuda(e);
+}
+
+moin_status moin_device_status_reset(moin_stream stream) {
+  HostState* hs;
+  moin_status st = host_state(&hs);
+  if (st) return st;
+  return record_cuda(cudaMemsetAsync(hs->status, 0, sizeof(DeviceStatus), (cudaStream_t)stream));
+}
+
+moin_status moin_profile_enable(int32_t capacity) {
+  if (capacity < 0) return MOIN_ERR_INVALID_ARG;
+  for (int i = 0; i < g_prof.capacity; ++i) {
+    cudaEventDestroy(g_prof.start[i]);
+    cudaEventDestroy(g_prof.stop[i]);
+  }
+  delete[] g_prof.start; delete[] g_prof.stop; delete[] g_prof.kernel; delete[] g_prof.launches;
+  g_prof = ProfState();
+  if (capacity == 0) return MOIN_OK;
+  g_prof.start = new cudaEvent_t[capacity];
+  g_prof.stop = new cudaEvent_t[capacity];
+  g_prof.kernel = new int[capacity];
+  g_prof.launches = new int[capacity];
+  for (int i = 0; i < capacity; ++i) {
+    cudaError_t e = cudaEventCreate(&g_prof.start[i]);
+    if (e == cudaSuccess) e = cudaEventCreate(&g_prof.stop[i]);
+    if (e != cudaSuccess) return record_cuda(e);
+  }
+  g_prof.capacity = capacity;
+  return MOIN_OK;
+}
+
+moin_status moin_profile_read(moin_profile_record* out, int32_t capacity, int32_t* n) {
+  if (!n || capacity < 0 || (capacity > 0 && !out)) return MOIN_ERR_INVALID_ARG;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return record_cuda(e);
+  *n = g_prof.count;
+  for (int i = 0; i < g_prof.count && i < capacity; ++i) {
+    out[i].kernel = g_prof.kernel[i];
+    out[i].launches = g_prof.launches[i];
+    out[i].ms = 0.f;
+    cudaEventElapsedTime(&out[i].ms, g_prof.start[i], g_prof.stop[i]);
+  }
+  g_prof.count = 0;
+  return MOIN_OK;
+}
+
+const char* moin_kernel_name(int32_t k) {
+  static const char* names[MOIN_K_COUNT] = {"route_simple", "route_tc", "route_finish", "plan", "gemm_warp", "gemm_tc",
+                                            "lora_shrink_stream", "lora_expand_stream", "lora_shrink_tc",
+                                            "lora_fused_tc", "decoder_glue", "attention"};
+  return (k >= 0 && k < MOIN_K_COUNT) ? names[k] : "unknown";
+}
+
+/* ------------------------------------------------------------------ router */
+
+moin_status moin_router_prepare(const void* centroids, int32_t K, int32_t D, float* inv_norm, moin_stream stream) {
+  if (!centroids || !inv_norm || K < 1) return MOIN_ERR_INVALID_ARG;
+  if (D < 8 || D > 8192 || (D % 8) != 0) return MOIN_ERR_BAD_SHAPE;
+  if (!aligned16(centroids)) return MOIN_ERR_MISALIGNED;
+  HostState* hs;
+  moin_status st = host_state(&hs);
+  if (st) return st;
+  ProfScope prof(MOIN_K_GLUE, 1, (cudaStream_t)stream);
+  return record_cuda(launch_inv_norm((const __nv_bfloat16*)centroids, K, D, inv_norm, (cudaStream_t)stream));
+}
+
+size_t moin_route_workspace_bytes(int32_t Q, int32_t K, int32_t D) {
+  (void)K; (void)D;
+  return align_up((size_t)(Q > 0 ? Q : 0) * sizeof(unsigned long long), 256) + 256;
+}
+
+moin_status moin_route(const moin_router* router, const void* queries, int32_t Q, int32_t* out_expert,
+                       int32_t* out_centroid, float* out_best_sim, void* workspace, size_t workspace_bytes,
+                       moin_stream stream) {
+  if (!router || Q < 0) return MOIN_ERR_INVALID_ARG;
+  if (Q == 0) return MOIN_OK;
+  if (!queries || !out_expert || !router->centroids || !router->inv_norm || router->K < 1) return MOIN_ERR_INVALID_ARG;
+  const int K = router->K, D = router->D;
+  if (D < 8 || D > 8192 || (D % 8) != 0) return MOIN_ERR_BAD_SHAPE;
+  if (!aligned16(queries) || !aligned16(router->centroids)) return MOIN_ERR_MISALIGNED;
+  HostState* hs;
+  moin_status st = host_state(&hs);
+  if (st) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  const bool tc_ok = tc_router_supported(Q, K, D);
+  bool use_tc = tc_ok && (long long)Q * K >= (1ll << 16);
+  if (hs->gemm_impl == 1) use_tc = false;
+  if (hs->gemm_impl == 2) {
+    if (!tc_ok) return MOIN_ERR_BAD_SHAPE;
+    use_tc = true;
+  }
+  if (use_tc) {
+    if (!workspace || workspace_bytes < moin_route_workspace_bytes(Q, K, D) || !aligned16(workspace))
+      return MOIN_ERR_WORKSPACE;
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(workspace);
+    cudaError_t e = cudaMemsetAsync(keys, 0, (size_t)Q * sizeof(unsigned long long), s);
+    if (e != cudaSuccess) return record_cuda(e);
+    {
+      ProfScope prof(MOIN_K_ROUTE_TC, 1, s);
+      st = launch_tc_router(hs, (const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids,
+                            router->inv_norm, Q, K, D, keys, s);
+    }
+    if (st) return st;
+    ProfScope prof(MOIN_K_ROUTE_FINISH, 1, s);
+    return record_cuda(launch_route_finish(keys, (const __nv_bfloat16*)queries, router->centroid_to_expert, Q, D,
+                                           out_expert, out_centroid, out_best_sim, s));
+  }
+  ProfScope prof(MOIN_K_ROUTE_SIMPLE, 1, s);
+  return record_cuda(launch_route_simple((const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids,
+                                         router->inv_norm, router->centroid_to_expert, Q, K, D, out_expert,
+                                         out_centroid, out_best_sim, s));
+}
+
+/* ------------------------------------------------------------------ plan */
+
+size_t moin_plan_bytes(int32_t T, int32_t E) {
+  if (T < 0 || E < 0) return 0;
+  return align_up(plan_bytes(T, E), 256);
+}
+
+moin_status moin_plan_build(const int32_t* token_expert, moin_plan* plan, moin_stream stream) {
+  if (!plan || plan->T < 0 || plan->E < 1) return MOIN_ERR_INVALID_ARG;
+  if (plan->mode < MOIN_PLAN_AUTO || plan->mode > MOIN_PLAN_TILES) return MOIN_ERR_INVALID_ARG;
+  if (plan->T == 0) return MOIN_OK;
+  if (!token_expert || !plan->buffer) return MOIN_ERR_INVALID_ARG;
+  if (!aligned16(plan->buffer)) return MOIN_ERR_MISALIGNED;
+  if (plan->buffer_bytes < plan_bytes(plan->T, plan->E)) return MOIN_ERR_WORKSPACE;
+  HostState* hs;
+  moin_status st = host_state(&hs);
+  if (st) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  PlanView v = plan_view(plan->buffer, plan->T, plan->E);
+  {
+    ProfScope prof(MOIN_K_PLAN, 3, s);
+    st = record_cuda(launch_plan_build(token_expert, v, hs->status, s));
+  }
+  if (st) return st;
+  if (plan->mode == MOIN_PLAN_AUTO) {
+    int header[kPlanHeaderWords];
+    cudaError_t e = cudaMemcpyAsync(header, v.header, sizeof(header), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return record_cuda(e);
+    plan->n_segments = header[PH_NSEG];
+    plan->n_tiles = header[PH_NTILES];
+    plan->n_lora_tokens = header[PH_NLORA];
+    plan->max_segment = header[PH_MAXSEG];
+    // Long runs (few, well-filled 128-row tiles) -> fold the adapter into the tensor-core GEMM.
+    const int full_tiles = (plan->T + kTileRows - 1) / kTileRows;
+    plan->mode = (plan->T >= 2 * kTileRows && plan->n_tiles <= full_tiles + full_tiles / 2) ? MOIN_PLAN_TILES
+                                                                                         : MOIN_PLAN_SEGMENTS;
+  }
+  return MOIN_OK;
+}
+
+moin_status moin_plan_read(const moin_plan* plan, int32_t* n_segments, int32_t* n_tiles, int32_t* perm,
+                           int32_t* seg_expert, int32_t* seg_start, int32_t* tile_row0, int32_t* tile_rows,
+                           int32_t* tile_expert, moin_stream stream) {
+  if (!plan || !plan->buffer || plan->T < 1) return MOIN_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  PlanView v = plan_view(plan->buffer, plan->T, plan->E);
+  int header[kPlanHeaderWords];
+  cudaError_t e = cudaMemcpyAsync(header, v.header, sizeof(header), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return record_cuda(e);
+  const int S = header[PH_NSEG], NT = header[PH_NTILES];
+  if (n_segments) *n_segments = S;
+  if (n_tiles) *n_tiles = NT;
+  auto copy = [&](int32_t* dst, const int* src, size_t n) {
+    if (dst && n && e == cudaSuccess) e = cudaMemcpyAsync(dst, src, n * sizeof(int), cudaMemcpyDeviceToHost, s);
+  };
+  copy(perm, v.perm, (size_t)plan->T);
+  copy(seg_expert, v.seg_expert, (size_t)S);
+  copy(seg_start, v.seg_start, (size_t)S + 1);
+  copy(tile_row0, v.tile_row0, (size_t)NT);
+  copy(tile_rows, v.tile_rows, (size_t)NT);
+  copy(tile_expert, v.tile_expert, (size_t)NT);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  return record_cuda(e);
+}
+
+/* ------------------------------------------------------------------ routed LoRA linear layer */
+
+size_t moin_lora_linear_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, int32_t r) {
+  (void)d_in;
+  if (T <= 0) return 256;
+  const size_t Tp = align_up((size_t)T, kTileRows) + kTileRows;
+  size_t seg = align_up((size_t)T * (size_t)(r > 0 ? r : 8) * sizeof(float), 256) +
+               align_up((size_t)T * (size_t)d_out * sizeof(float), 256);
+  size_t tiles = align_up(Tp * (size_t)64 * sizeof(__nv_bfloat16), 256);
+  return (seg > tiles ? seg : tiles) + 256;
+}
+
+moin_status moin_lora_linear(const moin_plan* plan, const void* x, const void* W, const moin_pool* pool,
+                             float scale, int32_t base_T, int32_t base_d_in, int32_t base_d_out, void* y,
+                             void* workspace, size_t workspace_bytes, moin_stream stream) {
+  const bool lora = (plan != nullptr && pool != nullptr);
+  const int T = lora ? plan->T : base_T;
+  const int d_in = lora ? pool->d_in : base_d_in;
+  const int d_out = lora ? pool->d_out : base_d_out;
+  if (T < 0) return MOIN_ERR_INVALID_ARG;
+  if (T == 0) return MOIN_OK;
+  if (!x || !W || !y || x == y) return MOIN_ERR_INVALID_ARG;
+  if (d_in < 64 || (d_in % 64) != 0 || d_out < 8 || (d_out % 8) != 0) return MOIN_ERR_BAD_SHAPE;
+  if (!aligned16(x) || !aligned16(W) || !aligned16(y)) return MOIN_ERR_MISALIGNED;
+  int r = 0;
+  if (lora) {
+    r = pool->r;
+    if (r < 8 || r > 64 || (r % 8) != 0) return MOIN_ERR_UNSUPPORTED_RANK;
+    if (!pool->A || !pool->B || !pool->slot_of_expert || !plan->buffer) return MOIN_ERR_INVALID_ARG;
+    if (pool->E != plan->E) return MOIN_ERR_INVALID_ARG;
+    if (!aligned16(pool->A) || !aligned16(pool->B)) return MOIN_ERR_MISALIGNED;
+    if (plan->mode != MOIN_PLAN_SEGMENTS && plan->mode != MOIN_PLAN_TILES) return MOIN_ERR_INVALID_ARG;
+  }
+  HostState* hs;
+  moin_status st = host_state(&hs);
+  if (st) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  const __nv_bfloat16* xb = (const __nv_bfloat16*)x;
+  const __nv_bfloat16* Wb = (const __nv_bfloat16*)W;
+  __nv_bfloat16* yb = (__nv_bfloat16*)y;
+
+  const bool tc_ok = tc_gemm_supported(T, d_in, d_out);
+  bool use_tc = tc_ok && T >= 64 && d_out >= 64;
+  if (hs->gemm_impl == 1) use_tc = false;
+  if (hs->gemm_impl == 2) {
+    if (!tc_ok) return MOIN_ERR_BAD_SHAPE;
+    use_tc = true;
+  }
+
+  if (!lora) {
+    ProfScope prof(use_tc ? MOIN_K_GEMM_TC : MOIN_K_GEMM_WARP, 1, s);
+    if (use_tc) return launch_tc_gemm(hs, xb, Wb, yb, nullptr, T, d_in, d_out, s);
+    return record_cuda(launch_gemm_warp(xb, Wb, yb, nullptr, T, d_in, d_out, s));
+  }
+  if (!workspace || !aligned16(workspace) || workspace_bytes < moin_lora_linear_workspace_bytes(T, d_in, d_out, r))
+    return MOIN_ERR_WORKSPACE;
+  PlanView pv = plan_view(plan->buffer, plan->T, plan->E);
+  char* ws = reinterpret_cast<char*>(workspace);
+
+  if (plan->mode == MOIN_PLAN_TILES && use_tc && tc_fused_supported(r)) {
+    __nv_bfloat16* hb = reinterpret_cast<__nv_bfloat16*>(ws);  // [T, r] bf16, s * (x A^T)
+    return launch_tc_lora_tiles(hs, pv, pool, xb, Wb, yb, hb, scale, s);
+  }
+  // Short segments: base GEMM (y and fp32 y0), then stream every distinct adapter once.
+  float* h = reinterpret_cast<float*>(ws);
+  float* y0 = reinterpret_cast<float*>(ws + align_up((size_t)T * (size_t)r * sizeof(float), 256));
+  {
+    ProfScope prof(use_tc ? MOIN_K_GEMM_TC : MOIN_K_GEMM_WARP, 1, s);
+    if (use_tc)
+      st = launch_tc_gemm(hs, xb, Wb, yb, y0, T, d_in, d_out, s);
+    else
+      st = record_cuda(launch_gemm_warp(xb, Wb, yb, y0, T, d_in, d_out, s));
+  }
+  if (st) return st;
+  {
+    ProfScope prof(MOIN_K_SHRINK_STREAM, 1, s);
+    st = record_cuda(launch_lora_shrink_stream(pv, pool->slot_of_expert, xb, (const __nv_bfloat16*)pool->A, h, r, d_in,
+                                               hs->n_sms, s));
+  }
+  if (st) return st;
+  ProfScope prof(MOIN_K_EXPAND_STREAM, 1, s);
+  return record_cuda(launch_lora_expand_stream(pv, pool->slot_of_expert, h, (const __nv_bfloat16*)pool->B, y0, yb,
+                                               scale, r, d_out, hs->n_sms, s));
+}
+
+}  // extern "C"

@@ -107,5 +107,37 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // Launchers implemented in the .cu files (host side).
 cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, DeviceStatus* status, cudaStream_t stream);
+cudaError_t launch_lora_shrink_stream(const PlanView& pv, const int* slot_of_expert, const __nv_bfloat16* x,
+                                      const __nv_bfloat16* A, float* h, int r, int d_in, int n_sms,
+                                      cudaStream_t stream);
+cudaError_t launch_lora_expand_stream(const PlanView& pv, const int* slot_of_expert, const float* h,
+                                      const __nv_bfloat16* B, const float* y0, __nv_bfloat16* y, float scale, int r,
+                                      int d_out, int n_sms, cudaStream_t stream);
+cudaError_t launch_gemm_warp(const __nv_bfloat16* x, const __nv_bfloat16* W, __nv_bfloat16* y, float* y0, int T,
+                             int d_in, int d_out, cudaStream_t stream);
+cudaError_t launch_inv_norm(const __nv_bfloat16* c, int K, int D, float* inv_norm, cudaStream_t stream);
+cudaError_t launch_route_simple(const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
+                                const int* cmap, int Q, int K, int D, int* out_expert, int* out_centroid,
+                                float* out_best, cudaStream_t stream);
+cudaError_t launch_route_finish(const unsigned long long* keys, const __nv_bfloat16* q, const int* cmap, int Q, int D,
+                                int* out_expert, int* out_centroid, float* out_best, cudaStream_t stream);
+
+// Process-wide host state shared by the entry points (api.cu).
+struct HostState {
+  DeviceStatus* status = nullptr;  // device address of the status block
+  int device = -1;
+  int n_sms = 0;
+  int gemm_impl = 0;               // MOIN_OPT_GEMM_IMPL
+};
+moin_status host_state(HostState** out);      // lazily initialised for the current device
+moin_status record_cuda(cudaError_t e);       // MOIN_OK or MOIN_ERR_CUDA (remembers e)
+
+// Brackets the launches issued during its lifetime with two CUDA events when profiling is enabled.
+struct ProfScope {
+  ProfScope(int kernel, int launches, cudaStream_t stream);
+  ~ProfScope();
+  int slot;
+  cudaStream_t stream;
+};
 
 }  // namespace moin

@@ -1,0 +1,102 @@
+"""Decoder forward on the GPU against the oracle (Llama-architecture blocks whose projections are routed
+LoRA layers).  Gate: block by block with the oracle's own block input (teacher forcing), and end to end
+against the oracle variant that rounds to bf16 where the library stores bf16; the distance to the pure
+fp64 oracle is printed."""
+import numpy as np
+import pytest
+import torch
+
+import moin_inputs as mi
+import oracle
+import paper_2410_09687_b200 as moin
+from gpu_util import DEV, REL_FRO
+
+pytestmark = pytest.mark.gpu
+
+CFG = mi.DecoderConfig(n_layers=3, hidden=256, n_heads=4, n_kv_heads=2, head_dim=64, ffn=512, vocab=1000,
+                       E=6, r=16, scale=2.0)
+
+
+def oracle_weights(model):
+    nl = model.cfg.n_layers
+    return {"embed": mi.bf16_bits(model.embed), "lm_head": mi.bf16_bits(model.lm_head),
+            "final_norm": mi.bf16_bits(model.final_norm),
+            "attn_norm": [mi.bf16_bits(t) for t in model.attn_norm],
+            "mlp_norm": [mi.bf16_bits(t) for t in model.mlp_norm],
+            "W": [{p: mi.bf16_bits(model.W[l][p]) for p in oracle.PROJ_ORDER} for l in range(nl)],
+            "A": [{p: mi.bf16_bits(model.pools[l][p].A) for p in oracle.PROJ_ORDER} for l in range(nl)],
+            "B": [{p: mi.bf16_bits(model.pools[l][p].B) for p in oracle.PROJ_ORDER} for l in range(nl)],
+            "slot_of_expert": model.pools[0]["q"].slot_of_expert.cpu().numpy()}
+
+
+def gpu_model(model):
+    nl = model.cfg.n_layers
+    pools = [{p: moin.Pool(model.pools[l][p].A.to(DEV), model.pools[l][p].B.to(DEV),
+                           model.pools[l][p].slot_of_expert.to(DEV)) for p in oracle.PROJ_ORDER} for l in range(nl)]
+    W = [{p: model.W[l][p].to(DEV) for p in oracle.PROJ_ORDER} for l in range(nl)]
+    return moin.DecoderModel(model.cfg, model.embed.to(DEV), model.lm_head.to(DEV), model.final_norm.to(DEV),
+                             [t.to(DEV) for t in model.attn_norm], [t.to(DEV) for t in model.mlp_norm], W, pools,
+                             model.cfg.E, model.cfg.scale)
+
+
+def rel(a, b):
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30))
+
+
+@pytest.fixture(scope="module")
+def setup():
+    model = mi.decoder_model(CFG, seed=4, missing=(2,))
+    return model, gpu_model(model), oracle.DecoderOracle(CFG, oracle_weights(model))
+
+
+@pytest.mark.parametrize("lengths,experts", [([70, 1, 129, 33, 64], [0, 2, 3, -1, 5]),      # short requests: segments
+                                             ([200, 130, 257], [1, 1, 4])])                 # long runs: tiles
+def test_decoder_end_to_end_and_block_by_block(setup, lengths, experts):
+    model, gm, orc = setup
+    batch = mi.decoder_batch(CFG, lengths, seed=4, req_expert=experts)
+    tok, cu, re_ = batch.tokens.to(DEV), batch.cu_seqlens.to(DEV), batch.req_expert.to(DEV)
+    args = (batch.tokens.numpy(), batch.cu_seqlens.numpy(), batch.req_expert.numpy())
+    hid = torch.empty(batch.T, CFG.hidden, dtype=torch.float32, device=DEV)
+    logits = moin.decoder_forward(gm, tok, cu, re_, max(lengths), hidden_out=hid)
+    torch.cuda.synchronize()
+    got = logits.to(torch.float64).cpu().numpy()
+    assert np.isfinite(got).all()
+    exact = orc.forward(*args)["logits"]
+    rounded = orc.forward(*args, round_storage=True, want_hidden=True)
+    e_exact, e_round = rel(got, exact), rel(got, rounded["logits"])
+    print(f"logits rel Frobenius: vs fp64 oracle {e_exact:.2e}, vs storage-rounded oracle {e_round:.2e}")
+    assert e_round <= REL_FRO
+    assert e_exact <= 4 * REL_FRO
+    assert rel(hid.double().cpu().numpy(), rounded["hidden"]) <= REL_FRO
+    # block by block: feed the GPU block the oracle's (storage-rounded) block input
+    h_in = orc.forward(*args, layer_begin=0, layer_end=0, want_hidden=True, want_logits=False)["hidden"]
+    for l in range(CFG.n_layers):
+        ref = orc.forward(*args, layer_begin=l, layer_end=l + 1, round_storage=True, hidden_in=h_in,
+                          want_hidden=True, want_logits=False)["hidden"]
+        hin_gpu = torch.from_numpy(h_in).to(torch.float32).to(DEV)
+        moin.decoder_forward(gm, tok, cu, re_, max(lengths), logits_mode=moin.LOGITS_NONE, hidden_in=hin_gpu,
+                             hidden_out=hid, layer_begin=l, layer_end=l + 1)
+        torch.cuda.synchronize()
+        d = hid.double().cpu().numpy() - h_in.astype(np.float32).astype(np.float64)
+        d_ref = ref - h_in
+        assert rel(d, d_ref) <= REL_FRO, f"block {l}"
+        h_in = ref
+
+
+def test_decoder_last_token_logits_and_request_independence(setup):
+    model, gm, orc = setup
+    lengths, experts = [40, 7, 90], [3, 0, -1]
+    batch = mi.decoder_batch(CFG, lengths, seed=5, req_expert=experts)
+    tok, cu, re_ = batch.tokens.to(DEV), batch.cu_seqlens.to(DEV), batch.req_expert.to(DEV)
+    full = moin.decoder_forward(gm, tok, cu, re_, 90)
+    last = moin.decoder_forward(gm, tok, cu, re_, 90, logits_mode=moin.LOGITS_LAST)
+    torch.cuda.synchronize()
+    cuh = batch.cu_seqlens.numpy()
+    assert torch.equal(last, full[torch.from_numpy(cuh[1:] - 1).long().to(DEV)])
+    # a request alone gives the same logits as inside the batch (introvert experts)
+    for r in range(3):
+        one = moin.decoder_forward(gm, tok[cuh[r]:cuh[r + 1]].contiguous(),
+                                   torch.tensor([0, lengths[r]], dtype=torch.int32, device=DEV),
+                                   re_[r:r + 1].contiguous(), lengths[r])
+        ref = full[cuh[r]:cuh[r + 1]].double()
+        assert float((one.double() - ref).norm() / ref.norm()) <= REL_FRO

@@ -1,0 +1,135 @@
+"""Routed LoRA linear layer on the GPU against the fp64 oracle (Sec. 3.2 formula, expert per token)."""
+import numpy as np
+import pytest
+import torch
+
+import moin_inputs as mi
+import oracle
+import paper_2410_09687_b200 as moin
+from gpu_util import DEV, assert_layer_close, gpu_pool, oracle_layer, run_layer
+
+pytestmark = pytest.mark.gpu
+MODES = [moin.PLAN_SEGMENTS, moin.PLAN_TILES]
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("impl", [0, 1])
+def test_tiny_config(mode, impl):
+    moin.set_option(moin.OPT_GEMM_IMPL, impl)
+    try:
+        case = mi.tiny_layer(seed=0)
+        y, _ = run_layer(case, mode)
+        assert_layer_close(y, oracle_layer(case), "tiny")
+    finally:
+        moin.set_option(moin.OPT_GEMM_IMPL, 0)
+
+
+def test_tiny_config_routed_by_the_router():
+    # the router's ids feed the layer: 16 requests, each routed to one of 8 experts
+    rc = mi.tiny_router(seed=0)
+    case = mi.tiny_layer(seed=0)
+    router = moin.Router(rc.centroids.to(DEV))
+    req_expert = moin.route(router, rc.queries.to(DEV)).cpu().numpy()
+    ref_ids = oracle.route(mi.bf16_bits(rc.queries), mi.bf16_bits(rc.centroids))["expert"]
+    assert np.array_equal(req_expert, ref_ids)
+    case.token_expert = torch.from_numpy(mi.expand_request_experts(req_expert, case.lengths))
+    y, _ = run_layer(case)
+    assert_layer_close(y, oracle_layer(case), "tiny routed")
+
+
+@pytest.mark.parametrize("r", [8, 16, 24, 32, 40, 48, 56, 64])
+@pytest.mark.parametrize("mode", MODES)
+def test_every_supported_rank(r, mode):
+    rng = mi.np_rng(7, r)
+    E, T, d_in, d_out = 6, 333, 192, 328     # ragged T, d_out not a multiple of 16 or 64
+    pool = mi.make_pool(E, r, d_in, d_out, 7, r, missing=(4,))
+    lens = rng.multinomial(T - 8, [1 / 8] * 8) + 1
+    te = np.repeat(rng.integers(-1, E, size=8), lens).astype(np.int32)
+    case = mi.layer_case("ranks", T, d_in, d_out, pool, te, 2.0, 7, r)
+    y, _ = run_layer(case, mode)
+    assert_layer_close(y, oracle_layer(case), f"rank {r}")
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_base_only_and_missing_adapters(mode):
+    pool = mi.make_pool(5, 16, 256, 128, 8, 1, missing=(1, 3))
+    te = np.array([-1, 1, 3, 0, 2, 4, 99, -5] * 20, np.int32)
+    case = mi.layer_case("fallback", len(te), 256, 128, pool, te, 2.0, 8, 2)
+    y, _ = run_layer(case, mode)
+    ref = oracle_layer(case)
+    assert_layer_close(y, ref, "fallback")
+    # tokens without an adapter equal the base layer computed by the same library
+    y_base = moin.lora_linear(None, case.x.to(DEV), case.W.to(DEV), None, 0.0)
+    so = pool.slot_of_expert.numpy()
+    base_rows = np.array([not (0 <= e < 5 and so[e] >= 0) for e in te])
+    assert torch.equal(y[torch.from_numpy(base_rows).to(DEV)], y_base[torch.from_numpy(base_rows).to(DEV)])
+    assert_layer_close(y_base, oracle.lora_linear(mi.bf16_bits(case.x), mi.bf16_bits(case.W), None, None, None,
+                                                  None, 0.0), "base")
+
+
+def test_decode_config_all_projections():
+    # 256 single-token requests, 500 rank-64 experts: every token checked against the oracle.
+    cases = mi.decode_batch(seed=1, device=DEV)
+    te = cases[0].token_expert
+    plan = moin.plan_build(te.to(DEV), 500, moin.PLAN_SEGMENTS)
+    for case in cases:
+        y, _ = run_layer(case, plan=plan)
+        rel = assert_layer_close(y, oracle_layer(case), f"decode {case.name}")
+        print(f"decode {case.name}: rel Frobenius {rel:.2e}")
+    del cases
+    torch.cuda.empty_cache()
+
+
+def test_prefill_config_sampled_rows():
+    # 32 x 512 tokens, 5 000 rank-16 experts, Zipf-skewed: 64 seeded rows per projection against the oracle.
+    cases = mi.prefill_batch(seed=2, device=DEV)
+    plan = moin.plan_build(cases[0].token_expert.to(DEV), 5000, moin.PLAN_AUTO)
+    rows = np.sort(np.random.default_rng(0).choice(cases[0].T, size=64, replace=False))
+    for case in cases:
+        y, _ = run_layer(case, plan=plan)
+        ref = oracle_layer(case, rows)
+        assert_layer_close(y[torch.from_numpy(rows).to(DEV)], ref, f"prefill {case.name}")
+    del cases
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_request_permutation_and_determinism(mode):
+    # experts do not interact: permuting requests permutes output rows (bitwise), and reruns are bitwise equal
+    pool = mi.make_pool(12, 32, 256, 256, 9, 1)
+    rng = mi.np_rng(9, 2)
+    req = rng.integers(0, 12, size=10)
+    L = 160
+    te = np.repeat(req, L).astype(np.int32)
+    case = mi.layer_case("perm", len(te), 256, 256, pool, te, 2.0, 9, 3)
+    gp = gpu_pool(pool)
+    y1, _ = run_layer(case, mode, pool=gp)
+    y2, _ = run_layer(case, mode, pool=gp)
+    assert torch.equal(y1, y2)
+    p = rng.permutation(10)
+    rows = np.concatenate([np.arange(i * L, (i + 1) * L) for i in p])
+    case_p = mi.LayerCase("perm2", case.x[torch.from_numpy(rows)], case.W, pool, torch.from_numpy(te[rows]), 2.0,
+                          len(te))
+    y3, _ = run_layer(case_p, mode, pool=gp)
+    assert torch.equal(y3, y1[torch.from_numpy(rows).to(DEV)])
+
+
+def test_empty_batch_and_argument_errors():
+    pool = gpu_pool(mi.make_pool(4, 8, 64, 64, 10, 1))
+    x = torch.zeros(0, 64, dtype=torch.bfloat16, device=DEV)
+    W = torch.zeros(64, 64, dtype=torch.bfloat16, device=DEV)
+    plan = moin.plan_build(torch.zeros(0, dtype=torch.int32, device=DEV), 4, moin.PLAN_SEGMENTS)
+    assert moin.lora_linear(plan, x, W, pool, 1.0).shape == (0, 64)
+    bad = moin.Pool(torch.zeros(4, 12, 64, dtype=torch.bfloat16, device=DEV),
+                    torch.zeros(4, 64, 12, dtype=torch.bfloat16, device=DEV), pool.slot_of_expert)
+    x1 = torch.zeros(8, 64, dtype=torch.bfloat16, device=DEV)
+    plan1 = moin.plan_build(torch.zeros(8, dtype=torch.int32, device=DEV), 4, moin.PLAN_SEGMENTS)
+    with pytest.raises(moin.MoinError, match="UNSUPPORTED_RANK"):
+        moin.lora_linear(plan1, x1, W, bad, 1.0)
+    with pytest.raises(moin.MoinError, match="BAD_SHAPE"):
+        moin.lora_linear(None, torch.zeros(8, 40, dtype=torch.bfloat16, device=DEV),
+                         torch.zeros(64, 40, dtype=torch.bfloat16, device=DEV), None, 1.0)
+    with pytest.raises(moin.MoinError, match="MISALIGNED"):
+        buf = torch.zeros(8 * 64 + 8, dtype=torch.bfloat16, device=DEV)
+        moin.lora_linear(None, buf[1:1 + 8 * 64].view(8, 64), W, None, 1.0)
+    assert moin.device_status()["timeout_flag"] == 0

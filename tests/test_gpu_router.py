@@ -1,0 +1,103 @@
+"""Router on the GPU against the oracle: ids bit-exact except near-ties (margin < 1e-4), which are counted."""
+import numpy as np
+import pytest
+import torch
+
+import moin_inputs as mi
+import oracle
+import paper_2410_09687_b200 as moin
+from gpu_util import DEV, TIE_MARGIN, assert_router_matches
+
+pytestmark = pytest.mark.gpu
+
+
+def _route(case: mi.RouterCase, cmap=None, impl=0):
+    moin.set_option(moin.OPT_GEMM_IMPL, impl)
+    try:
+        c, q = case.centroids.to(DEV), case.queries.to(DEV)
+        m = None if cmap is None else torch.from_numpy(cmap).to(DEV)
+        router = moin.Router(c, m)
+        cid = torch.empty(case.Q, dtype=torch.int32, device=DEV)
+        best = torch.empty(case.Q, dtype=torch.float32, device=DEV)
+        eid = moin.route(router, q, out_centroid=cid, out_best_sim=best)
+        torch.cuda.synchronize()
+        return eid.cpu().numpy(), cid.cpu().numpy(), best.cpu().numpy()
+    finally:
+        moin.set_option(moin.OPT_GEMM_IMPL, 0)
+
+
+def _oracle(case, cmap=None, rows=None):
+    q = mi.bf16_bits(case.queries if rows is None else case.queries[torch.as_tensor(rows)])
+    return oracle.route(q, mi.bf16_bits(case.centroids), cmap)
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_router_tiny(impl):
+    case = mi.tiny_router(seed=0)
+    eid, cid, best = _route(case, impl=impl)
+    ref = _oracle(case)
+    assert_router_matches(cid, ref)
+    assert np.array_equal(eid, cid)
+    np.testing.assert_allclose(best, ref["best"], atol=2e-3)
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_router_decode_shape_with_map(impl):
+    case = mi.planted_router(K=500, Q=256, D=768, seed=1)
+    cmap = np.arange(500, dtype=np.int32)[::-1].copy()
+    cmap[::7] = -1
+    eid, cid, best = _route(case, cmap, impl=impl)
+    ref = _oracle(case, cmap)
+    assert_router_matches(cid, ref)
+    assert np.array_equal(eid, cmap[cid])
+    assert np.array_equal(cid, case.labels.numpy())
+    np.testing.assert_allclose(best, ref["best"], atol=2e-3)
+
+
+def test_router_prefill_shape_5000_centroids():
+    case = mi.planted_router(K=5000, Q=32, D=768, seed=2)
+    _, cid, _ = _route(case)
+    assert_router_matches(cid, _oracle(case))
+
+
+def test_router_stress_full_size_sampled():
+    # 65 536 x 5 000 x 768 on the GPU; the oracle checks a seeded sample of queries one by one.
+    case = mi.planted_router(K=5000, Q=65536, D=768, seed=3, device=DEV)
+    _, cid, _ = _route(case)
+    assert np.array_equal(cid, case.labels.cpu().numpy())     # planted label (property at any size)
+    rows = np.random.default_rng(0).choice(65536, size=1024, replace=False)
+    host = mi.RouterCase(case.centroids.cpu(), case.queries.cpu(), None, case.K, case.D, case.Q)
+    ref = _oracle(host, rows=rows)
+    assert_router_matches(cid[rows], ref)
+
+
+def test_router_near_tie_stress():
+    # noise added to the UNIT centroid: many small margins; mismatches only allowed below the margin.
+    case = mi.planted_router(K=1000, Q=2048, D=768, seed=5, unit_centroid_noise=True)
+    _, cid, _ = _route(case)
+    ref = _oracle(case)
+    n_near, n_diff = assert_router_matches(cid, ref)
+    print(f"near-ties (<{TIE_MARGIN}): {n_near}, of which differ: {n_diff}")
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_router_degenerate_inputs(impl):
+    rng = np.random.default_rng(6)
+    c = torch.from_numpy(rng.normal(size=(70, 64))).to(torch.bfloat16)
+    c[3] = 0                       # zero-norm centroid: never chosen
+    c[50] = c[10] * 4              # same direction as 10: exact tie in cosine up to rounding -> lowest index
+    q = torch.from_numpy(rng.normal(size=(33, 64))).to(torch.bfloat16)
+    q[0] = c[10]
+    q[1] = c[3]                    # zero query
+    case = mi.RouterCase(c, q, None, 70, 64, 33)
+    _, cid, _ = _route(case, impl=impl)
+    ref = _oracle(case)
+    assert_router_matches(cid, ref)
+    assert cid[0] in (10, 50) and cid[1] == 0 and 3 not in cid[2:]
+
+
+def test_router_empty_batch():
+    case = mi.tiny_router(seed=0)
+    router = moin.Router(case.centroids.to(DEV))
+    out = moin.route(router, torch.empty(0, 64, dtype=torch.bfloat16, device=DEV))
+    assert out.numel() == 0
