@@ -1,0 +1,669 @@
+#!/usr/bin/env python
+"""Benchmark of the MoIN serving hot path on B200 (one JSON line on stdout).
+
+A "step" is one pass of the whole hot path over one batch of synthetic input:
+  decode  (default): route 256 query embeddings over 500 centroids -> batch plan -> the seven
+           TinyLlama-shaped projections with 500 rank-64 experts resident in HBM (256 single tokens)
+  prefill: route 32 queries over 5 000 centroids -> plan -> seven projections, 32 x 512 tokens,
+           5 000 rank-16 experts, Zipf(1.1) request experts
+  router:  65 536 queries x 5 000 centroids x 768
+  forward: 22-block decoder, 64 x 256 tokens, 500 rank-64 experts on all seven projections
+
+`value` is device-timed throughput with inputs resident in HBM; `e2e` repeats the measurement
+with host buffers (pinned host -> device copies of the step's inputs and a device -> host copy of
+its outputs inside the timed region).  `roofline` times the dominant kernel with CUDA events
+inside the library; `cpu_baseline` times the CPU oracle on a bounded sample of the same work.
+`--impl reference` times that oracle alone.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import moin_inputs as mi
+
+NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
+FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
+ROTATE = 4  # distinct input batches rotated through the timed steps
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        self.lines = []
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            sel = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            sel = str(device_index)
+        self.cmd = ["nvidia-smi", "-i", sel, f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"]
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(self.cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no_samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------------
+# workloads
+# ----------------------------------------------------------------------------------------------
+class LayerWorkload:
+    """route -> plan -> seven projections.  decode: E=500 r=64 T=256; prefill: E=5000 r=16 32x512."""
+
+    def __init__(self, kind: str, dev: str):
+        import paper_2410_09687_b200 as moin
+        self.moin, self.kind, self.dev = moin, kind, dev
+        if kind == "decode":
+            self.E, self.r, self.T, self.R, self.K, self.seed = 500, 64, 256, 256, 500, 1
+            self.mode = moin.PLAN_SEGMENTS
+        else:
+            self.E, self.r, self.T, self.R, self.K, self.seed = 5000, 16, 16384, 32, 5000, 2
+            self.mode = moin.PLAN_TILES
+        self.D, self.scale = 768, 2.0
+        self.unit, self.units_per_step = "tokens", self.T
+        self.projs = mi.TINYLLAMA_PROJECTIONS
+        # resident state: centroid table, adapter pools, base weights
+        rc = mi.planted_router(self.K, self.R * ROTATE, self.D, self.seed, device=dev)
+        self.router = moin.Router(rc.centroids)
+        self.queries = [rc.queries[i * self.R:(i + 1) * self.R].contiguous() for i in range(ROTATE)]
+        self.labels = [rc.labels[i * self.R:(i + 1) * self.R] for i in range(ROTATE)]
+        if kind == "prefill":   # Zipf-skewed request experts: planted labels -> skewed expert ids via the map
+            cmaps = []
+            for i in range(ROTATE):
+                z = mi.zipf_experts(self.R, self.E, 1.1, self.seed, 21 + i)
+                cmap = np.arange(self.K, dtype=np.int32)
+                cmap[self.labels[i].cpu().numpy()] = z     # centroid of request j -> Zipf expert of request j
+                cmaps.append(torch.from_numpy(cmap).to(dev))
+            self.routers = [moin.Router(rc.centroids, m) for m in cmaps]
+        else:
+            self.routers = [self.router] * ROTATE
+        self.pools, self.W, self.x, self.y = [], [], [], []
+        for p, (name, d_in, d_out) in enumerate(self.projs):
+            pool = mi.make_pool(self.E, self.r, d_in, d_out, self.seed, 30 + p, device=dev)
+            self.pools.append(moin.Pool(pool.A, pool.B, pool.slot_of_expert))
+            self.W.append(mi.normal_bf16((d_out, d_in), 0.02, self.seed, 40 + p, 12, device=dev))
+            self.x.append([mi.normal_bf16((self.T, d_in), 1.0, self.seed, 40 + p, 11, i, device=dev)
+                           for i in range(ROTATE)])
+            self.y.append(torch.empty(self.T, d_out, dtype=torch.bfloat16, device=dev))
+        self.req_expert = torch.empty(self.R, dtype=torch.int32, device=dev)
+        self.token_expert = torch.empty(self.T, dtype=torch.int32, device=dev)
+        self.plan = moin.Plan(self.T, self.E, dev, self.mode)
+        ws = max(moin.lib().moin_lora_linear_workspace_bytes(self.T, d_in, d_out, self.r) for _, d_in, d_out in self.projs)
+        self.ws = torch.empty(ws, dtype=torch.uint8, device=dev)
+        # host-side staging for the end-to-end arm
+        self.n_host = ROTATE if kind == "decode" else 1
+        self.h_q = [q.cpu().pin_memory() for q in self.queries[:self.n_host]]
+        self.h_x = [[x.cpu().pin_memory() for x in xs[:self.n_host]] for xs in self.x]
+        self.h_y = [torch.empty_like(y, device="cpu").pin_memory() for y in self.y]
+        self.d_q = torch.empty_like(self.queries[0])
+        self.d_x = [torch.empty_like(xs[0]) for xs in self.x]
+        self.h2d = self.d_q.numel() * 2 + sum(x.numel() * 2 for x in self.d_x)
+        self.d2h = sum(y.numel() * 2 for y in self.y)
+
+    def _core(self, i: int, q, xs):
+        moin = self.moin
+        moin.route(self.routers[i], q, out_expert=self.req_expert)
+        if self.kind == "decode":
+            te = self.req_expert
+        else:
+            L = self.T // self.R   # plumbing: request id -> its tokens
+            self.token_expert.view(self.R, L).copy_(self.req_expert.unsqueeze(1).expand(self.R, L))
+            te = self.token_expert
+        moin.plan_build(te, self.E, self.mode, plan=self.plan)
+        for p in range(len(self.projs)):
+            moin.lora_linear(self.plan, xs[p], self.W[p], self.pools[p], self.scale, y=self.y[p], workspace=self.ws)
+
+    def step(self, i: int):
+        i %= ROTATE
+        self._core(i, self.queries[i], [xs[i] for xs in self.x])
+
+    def step_e2e(self, i: int):
+        i %= ROTATE
+        j = i % self.n_host
+        self.d_q.copy_(self.h_q[j], non_blocking=True)
+        for p in range(len(self.projs)):
+            self.d_x[p].copy_(self.h_x[p][j], non_blocking=True)
+        self._core(i, self.d_q, self.d_x)
+        for p in range(len(self.projs)):
+            self.h_y[p].copy_(self.y[p], non_blocking=True)
+
+    def distinct(self) -> float:
+        vals = []
+        for i in range(ROTATE):
+            self.moin.route(self.routers[i], self.queries[i], out_expert=self.req_expert)
+            vals.append(int(torch.unique(self.req_expert[self.req_expert >= 0]).numel()))
+        return float(np.mean(vals))
+
+    def algorithmic(self, n_distinct: float) -> dict:
+        """Bytes / flops one step must move or compute: x, W, y once; every distinct adapter once."""
+        T, r = self.T, self.r
+        per = {"gemm": 0.0, "shrink": 0.0, "expand": 0.0}
+        flops = 0.0
+        for _, d_in, d_out in self.projs:
+            per["gemm"] += d_out * d_in * 2 + T * d_in * 2 + T * d_out * 2
+            per["shrink"] += n_distinct * r * d_in * 2 + T * d_in * 2 + T * r * 4
+            per["expand"] += n_distinct * d_out * r * 2 + T * r * 4 + T * d_out * 2
+            flops += 2.0 * T * d_in * d_out + 2.0 * T * r * (d_in + d_out)
+        step_bytes = sum((d_out * d_in + T * d_in + T * d_out + n_distinct * r * (d_in + d_out)) * 2
+                         for _, d_in, d_out in self.projs) + self.R * self.D * 2 + self.K * self.D * 2
+        return {"per_kernel_bytes": per, "step_bytes": step_bytes, "step_flops": flops}
+
+    def config(self) -> dict:
+        name = ("decode: 7 TinyLlama projections, 500 experts rank 64, 256 single tokens, router 256x500x768"
+                if self.kind == "decode" else
+                "prefill: 7 TinyLlama projections, 5000 experts rank 16, 32x512 tokens Zipf(1.1), router 32x5000x768")
+        return {"workload": name, "tokens_per_step": self.T, "experts": self.E, "rank": self.r, "lora_scale": self.scale,
+                "l2": f"inputs rotate over {ROTATE} batches; per-step working set exceeds L2"}
+
+    def oracle_sample(self, n_tokens: int) -> float:
+        """Seconds the CPU oracle needs for route + the seven projections of the first n_tokens tokens of batch 0."""
+        import oracle
+        n_req = max(1, n_tokens * self.R // self.T)
+        rows = np.arange(n_tokens)
+        q = mi.bf16_bits(self.queries[0][:n_req])
+        c = mi.bf16_bits(self.router.centroids)
+        self.step(0)
+        torch.cuda.synchronize()
+        te = (self.req_expert if self.kind == "decode" else self.token_expert).cpu().numpy()[rows]
+        used = sorted(set(int(e) for e in te if e >= 0))
+        remap = np.full(self.E, -1, np.int32)
+        remap[used] = np.arange(len(used))
+        idx = torch.tensor(used, dtype=torch.long, device=self.dev)
+        host = []
+        for p, (_, d_in, d_out) in enumerate(self.projs):
+            host.append((mi.bf16_bits(self.x[p][0][:n_tokens]), mi.bf16_bits(self.W[p]),
+                         mi.bf16_bits(self.pools[p].A[idx]), mi.bf16_bits(self.pools[p].B[idx])))
+        t0 = time.perf_counter()
+        oracle.route(q, c)
+        for x, W, A, B in host:
+            oracle.lora_linear(x, W, A, B, te, remap, self.scale)
+        return time.perf_counter() - t0
+
+
+class RouterWorkload:
+    def __init__(self, dev: str, Q: int = 65536, K: int = 5000, D: int = 768):
+        import paper_2410_09687_b200 as moin
+        self.moin, self.dev, self.Q, self.K, self.D = moin, dev, Q, K, D
+        rc = mi.planted_router(K, Q, D, 3, device=dev)
+        self.router = moin.Router(rc.centroids)
+        # rotate by rolling the query matrix: same multiset of queries, different rows per buffer
+        self.queries = [rc.queries] + [torch.roll(rc.queries, shifts=i * 4099, dims=0).contiguous() for i in range(1, ROTATE)]
+        self.out = torch.empty(Q, dtype=torch.int32, device=dev)
+        self.unit, self.units_per_step = "queries", Q
+        self.h_q = [self.queries[0].cpu().pin_memory()]
+        self.h_out = torch.empty(Q, dtype=torch.int32).pin_memory()
+        self.d_q = torch.empty_like(rc.queries)
+        self.h2d, self.d2h = Q * D * 2, Q * 4
+
+    def step(self, i: int):
+        self.moin.route(self.router, self.queries[i % ROTATE], out_expert=self.out)
+
+    def step_e2e(self, i: int):
+        self.d_q.copy_(self.h_q[0], non_blocking=True)
+        self.moin.route(self.router, self.d_q, out_expert=self.out)
+        self.h_out.copy_(self.out, non_blocking=True)
+
+    def config(self) -> dict:
+        return {"workload": f"router stress: {self.Q} queries x {self.K} centroids x {self.D}, planted clusters",
+                "l2": f"query matrix (100.7 MB) rotates over {ROTATE} buffers (> L2 in total)"}
+
+    def algorithmic(self) -> dict:
+        return {"flops": 2.0 * self.Q * self.K * self.D, "bytes": (self.Q + self.K) * self.D * 2 + self.Q * 4}
+
+    def oracle_sample(self, n: int) -> float:
+        import oracle
+        q = mi.bf16_bits(self.queries[0][:n])
+        c = mi.bf16_bits(self.router.centroids)
+        t0 = time.perf_counter()
+        oracle.route(q, c)
+        return time.perf_counter() - t0
+
+
+class ForwardWorkload:
+    """22-block decoder, 64 x 256 tokens, 500 rank-64 experts on all 7 projections (pool ~50 GB)."""
+
+    def __init__(self, dev: str, n_layers: int = 22, R: int = 64, L: int = 256):
+        import paper_2410_09687_b200 as moin
+        self.moin, self.dev = moin, dev
+        cfg = mi.DecoderConfig(n_layers=n_layers)
+        self.cfg, self.R, self.L, self.T = cfg, R, L, R * L
+        model = mi.decoder_model(cfg, seed=4, device=dev)
+        order = ("q", "k", "v", "o", "gate", "up", "down")
+        pools = [{p: moin.Pool(model.pools[l][p].A, model.pools[l][p].B, model.pools[l][p].slot_of_expert)
+                  for p in order} for l in range(n_layers)]
+        self.gm = moin.DecoderModel(cfg, model.embed, model.lm_head, model.final_norm, model.attn_norm, model.mlp_norm,
+                                    [{p: model.W[l][p] for p in order} for l in range(n_layers)], pools, cfg.E, cfg.scale)
+        self.batches = [mi.decoder_batch(cfg, [L] * R, seed=4 + i, device=dev) for i in range(ROTATE)]
+        self.logits = torch.empty(self.T, cfg.vocab, dtype=torch.bfloat16, device=dev)
+        self.unit, self.units_per_step = "tokens", self.T
+        self.h_tok = [b.tokens.cpu().pin_memory() for b in self.batches]
+        self.d_tok = torch.empty_like(self.batches[0].tokens)
+        self.h_last = torch.empty(R, cfg.vocab, dtype=torch.bfloat16).pin_memory()
+        self.last = torch.empty(R, cfg.vocab, dtype=torch.bfloat16, device=dev)
+        self.h2d, self.d2h = self.T * 4, R * cfg.vocab * 2
+        self.gm.workspace(R, self.T)
+
+    def step(self, i: int):
+        b = self.batches[i % ROTATE]
+        self.moin.decoder_forward(self.gm, b.tokens, b.cu_seqlens, b.req_expert, self.L, logits=self.logits)
+
+    def step_e2e(self, i: int):
+        b = self.batches[i % ROTATE]
+        self.d_tok.copy_(self.h_tok[i % ROTATE], non_blocking=True)
+        self.moin.decoder_forward(self.gm, self.d_tok, b.cu_seqlens, b.req_expert, self.L,
+                                  logits_mode=self.moin.LOGITS_LAST, logits=self.last)
+        self.h_last.copy_(self.last, non_blocking=True)
+
+    def config(self) -> dict:
+        return {"workload": f"full decoder forward: {self.cfg.n_layers} TinyLlama-shaped blocks, {self.R}x{self.L} tokens, "
+                            f"500 experts rank 64 on 7 projections, all-position logits",
+                "l2": "activations and weights per step far exceed L2"}
+
+    def algorithmic(self) -> dict:
+        c, T = self.cfg, self.T
+        per_layer = sum(2.0 * T * d_in * d_out + 2.0 * T * c.r * (d_in + d_out) for _, d_in, d_out in c.projections())
+        attn = 2.0 * 2.0 * self.R * c.n_heads * (self.L * (self.L + 1) / 2) * c.head_dim
+        return {"flops": c.n_layers * (per_layer + attn) + 2.0 * T * c.hidden * c.vocab}
+
+
+# ----------------------------------------------------------------------------------------------
+# measurement helpers
+# ----------------------------------------------------------------------------------------------
+def dist_setup(n_gpus: int):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+        local = 0
+    return world, rank, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(world, v: float) -> float:
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([v], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+    return v
+
+
+def timed_loop(world, fn, steps: int, warmup: int, use_graph: bool) -> float:
+    """ms per step over exactly `steps` steps, CUDA events on the launching stream, barrier + sync both sides."""
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for i in range(max(warmup, 3)):
+            fn(i)
+        stream.synchronize()
+        graphs = None
+        if use_graph:
+            try:
+                graphs = []
+                for i in range(ROTATE):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=stream):
+                        fn(i)
+                    graphs.append(g)
+                for g in graphs:
+                    g.replay()
+                stream.synchronize()
+            except Exception as e:  # pragma: no cover
+                sys.stderr.write(f"[bench] CUDA graph capture failed ({e}); timing plain launches\n")
+                graphs = None
+                torch.cuda.synchronize()
+        barrier(world)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        if graphs is not None:
+            for i in range(steps):
+                graphs[i % ROTATE].replay()
+        else:
+            for i in range(steps):
+                fn(i)
+        e1.record(stream)
+        stream.synchronize()
+        barrier(world)
+        torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps, graphs is not None
+
+
+def profile_pass(moin, fn, steps: int):
+    """Per-kernel device time (CUDA events inside the library, on the launching stream)."""
+    moin.profile_enable(65536)
+    try:
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            fn(0)
+            stream.synchronize()
+            moin.profile_read()
+            for i in range(steps):
+                fn(i)
+            stream.synchronize()
+        recs = moin.profile_read()
+    finally:
+        moin.profile_enable(0)
+    agg = {}
+    for r in recs:
+        a = agg.setdefault(r["kernel"], {"launches": 0, "brackets": 0, "ms": 0.0})
+        a["launches"] += r["launches"]; a["brackets"] += 1; a["ms"] += r["ms"]
+    launches_per_step = sum(a["launches"] for a in agg.values()) / steps
+    return agg, launches_per_step
+
+
+def traffic_for(kernel: str, workload: str):
+    """DRAM bytes per launch from the committed ncu capture, or None when the kernel source changed since."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(p):
+        return None
+    try:
+        d = json.load(open(p)).get(f"{kernel}:{workload}")
+        if not d:
+            return None
+        src = os.path.join(ROOT, d["source"])
+        if hashlib.sha256(open(src, "rb").read()).hexdigest()[:16] != d["source_sha256_16"]:
+            return None
+        return d["dram_bytes_per_launch"]
+    except Exception:
+        return None
+
+
+def adaptive_oracle(sample_fn, first: int, cap: int, target_s: float = 12.0):
+    """Times the oracle on `first` units, then once more on a sample sized for ~target_s seconds."""
+    t = sample_fn(first)
+    n = int(min(cap, max(first, first * target_s / max(t, 1e-3))))
+    if n > first * 1.5:
+        t = sample_fn(n)
+    else:
+        n = first
+    return n, t
+
+
+# ----------------------------------------------------------------------------------------------
+def run_reference(args):
+    """Reference arm = the CPU oracle as it stands, on this machine's host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    oracle.build()
+    cores = oracle.num_threads()
+    kind = args.workload
+    rng_seed = {"decode": 1, "prefill": 2, "router": 3, "forward": 4}[kind]
+    if kind == "router":
+        n, K, D = 256, 5000, 768
+        rc = mi.planted_router(K, n, D, rng_seed)
+        q, c = mi.bf16_bits(rc.queries), mi.bf16_bits(rc.centroids)
+        fn = lambda: oracle.route(q, c)
+        unit, metric, sample = "queries/s", "router_queries_per_s", f"{n} of 65536 queries per step, all 5000 centroids"
+        cfgname = "router stress: 65536 queries x 5000 centroids x 768, planted clusters"
+    else:
+        if kind == "forward":
+            sys.stderr.write("[bench] reference arm for 'forward' times the seven projections of one block\n")
+        E, r, n = (500, 64, 32) if kind != "prefill" else (5000, 16, 32)
+        te = np.random.default_rng(rng_seed).integers(0, 8, size=n).astype(np.int32)
+        slot = np.full(E, -1, np.int32); slot[:8] = np.arange(8)
+        host = []
+        for p, (_, d_in, d_out) in enumerate(mi.TINYLLAMA_PROJECTIONS):
+            pool = mi.make_pool(8, r, d_in, d_out, rng_seed, 30 + p)
+            host.append((mi.bf16_bits(mi.normal_bf16((n, d_in), 1.0, rng_seed, 40 + p, 11)),
+                         mi.bf16_bits(mi.normal_bf16((d_out, d_in), 0.02, rng_seed, 40 + p, 12)),
+                         mi.bf16_bits(pool.A), mi.bf16_bits(pool.B)))
+        rc = mi.planted_router(500 if kind != "prefill" else 5000, n if kind == "decode" else 1, 768, rng_seed)
+        q, c = mi.bf16_bits(rc.queries), mi.bf16_bits(rc.centroids)
+
+        def fn():
+            oracle.route(q, c)
+            for x, W, A, B in host:
+                oracle.lora_linear(x, W, A, B, te, slot, 2.0)
+        unit, metric = "tokens/s", "routed_lora_tokens_per_s"
+        sample = f"{n} tokens per step through route + the 7 projections (8 distinct adapters)"
+        cfgname = {"decode": "decode: 7 TinyLlama projections, 500 experts rank 64, 256 single tokens, router 256x500x768",
+                   "prefill": "prefill: 7 TinyLlama projections, 5000 experts rank 16, 32x512 tokens Zipf(1.1), router 32x5000x768",
+                   "forward": "full decoder forward (projections of one block as the sample)"}[kind]
+    for _ in range(args.warmup):
+        fn()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        fn()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = n / dt
+    line = {"impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": cfgname},
+            "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="moin", choices=["moin", "reference"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "router", "forward"])
+    ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-router-extra", action="store_true")
+    ap.add_argument("--forward-layers", type=int, default=22)
+    args = ap.parse_args()
+    defaults = {"decode": (3000, 20), "prefill": (100, 5), "router": (50, 5), "forward": (5, 3)}
+    if args.impl == "reference":
+        args.steps = args.steps if args.steps is not None else 5
+        args.warmup = args.warmup if args.warmup is not None else 1
+        return run_reference(args)
+    if args.steps is None:
+        args.steps = defaults[args.workload][0]
+    if args.warmup is None:
+        args.warmup = defaults[args.workload][1]
+
+    import paper_2410_09687_b200 as moin
+    if not os.path.exists(moin.lib_path()):
+        from paper_2410_09687_b200 import build
+        build.build()
+    moin.lib()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    world, rank, local = dist_setup(args.gpus)
+    dev = f"cuda:{local}"
+    peaks = load_peaks()
+    kind = args.workload
+    if kind in ("decode", "prefill"):
+        wl = LayerWorkload(kind, dev)
+    elif kind == "router":
+        wl = RouterWorkload(dev)
+    else:
+        wl = ForwardWorkload(dev, n_layers=args.forward_layers)
+    torch.cuda.synchronize()
+    use_graph = (not args.no_graph) and kind != "forward"
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, graphed = timed_loop(world, wl.step, args.steps, args.warmup, use_graph)
+    clocks = sampler.stop()
+    ms = max_over_ranks(world, ms)
+    value = world * wl.units_per_step / (ms * 1e-3)
+
+    e2e_steps = max(5, args.steps // 4)
+    ms_e2e, _ = timed_loop(world, wl.step_e2e, e2e_steps, max(3, args.warmup // 2), use_graph)
+    ms_e2e = max_over_ranks(world, ms_e2e)
+
+    # per-kernel timing -> roofline of the dominant kernel
+    agg, launches_per_step = profile_pass(moin, wl.step, min(args.steps, 20))
+    top = max(agg.items(), key=lambda kv: kv[1]["ms"])[0]
+    total_ms = sum(a["ms"] for a in agg.values())
+    kernels = {k: {"launches": a["launches"], "ms_per_launch": a["ms"] / max(a["launches"], 1),
+                   "share": a["ms"] / total_ms} for k, a in agg.items()}
+    prof_steps = min(args.steps, 20)
+    roof = None
+    extra = {}
+    if kind in ("decode", "prefill"):
+        nd = wl.distinct()
+        alg = wl.algorithmic(nd)
+        t_hbm = alg["step_bytes"] / (peaks["hbm_gbs"] * 1e9)
+        t_tc = alg["step_flops"] / (peaks["bf16_tflops"] * 1e12)
+        bound_time = max(t_hbm, t_tc)
+        extra["step_roofline"] = {"bound": "hbm" if t_hbm >= t_tc else "tensor", "algorithmic_bytes": alg["step_bytes"],
+                                  "algorithmic_flops": alg["step_flops"], "roofline_ms": bound_time * 1e3,
+                                  "frac": bound_time * 1e3 / ms,
+                                  "frac_nominal": max(alg["step_bytes"] / (NOMINAL_HBM_GBS * 1e9),
+                                                      alg["step_flops"] / (NOMINAL_BF16_TFLOPS * 1e12)) * 1e3 / ms,
+                                  "distinct_experts": nd}
+        name_to_key = {"lora_expand_stream": "expand", "lora_shrink_stream": "shrink", "gemm_warp": "gemm", "gemm_tc": "gemm"}
+        if top in name_to_key:
+            a = agg[top]
+            bytes_per_launch = alg["per_kernel_bytes"][name_to_key[top]] / len(wl.projs)
+            sec = a["ms"] * 1e-3 / a["launches"]
+            ach = bytes_per_launch / sec / 1e9
+            roof = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": ach / peaks["hbm_gbs"], "frac_nominal": ach / NOMINAL_HBM_GBS, "peak_source": peaks["source"],
+                    "algorithmic_bytes_per_launch": bytes_per_launch, "avg_launch_ms": sec * 1e3,
+                    "traffic": traffic_for(top, kind)}
+        elif top in ("lora_fused_tc", "lora_shrink_tc"):
+            a = agg[top]
+            fl = alg["step_flops"] / len(wl.projs)
+            sec = a["ms"] * 1e-3 / a["launches"]
+            ach = fl / sec / 1e12
+            roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "frac_burst": ach / peaks["bf16_tflops"],
+                    "frac_nominal": ach / NOMINAL_BF16_TFLOPS, "peak_source": peaks["source"] + " (sustained)",
+                    "algorithmic_flops_per_launch": fl, "avg_launch_ms": sec * 1e3, "traffic": traffic_for(top, kind)}
+    elif kind == "router":
+        alg = wl.algorithmic()
+        a = agg[top]
+        sec = a["ms"] * 1e-3 / a["launches"]
+        ach = alg["flops"] / sec / 1e12
+        tensor = top == "route_tc"
+        roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops"], "frac_nominal": ach / NOMINAL_BF16_TFLOPS,
+                "peak_source": peaks["source"] + " (burst)", "algorithmic_flops_per_launch": alg["flops"],
+                "avg_launch_ms": sec * 1e3, "traffic": traffic_for(top, kind), "tensor_core_kernel": tensor}
+    else:
+        alg = wl.algorithmic()
+        ach = alg["flops"] / (ms * 1e-3) / 1e12
+        roof = {"kernel": "whole forward (" + top + " dominant)", "bound": "tensor", "achieved": ach,
+                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
+                "frac_nominal": ach / NOMINAL_BF16_TFLOPS, "peak_source": peaks["source"] + " (sustained)",
+                "algorithmic_flops_per_launch": alg["flops"], "avg_launch_ms": ms, "traffic": None}
+    if roof is None:
+        a = agg[top]
+        roof = {"kernel": top, "bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": None,
+                "traffic": None, "avg_launch_ms": a["ms"] / a["launches"]}
+
+    # secondary number of the metric: router queries/s on the router-stress configuration
+    if kind == "decode" and rank == 0 and not args.no_router_extra:
+        rw = RouterWorkload(dev)
+        rms, _ = timed_loop(1, rw.step, 10, 3, False)
+        ragg, _ = profile_pass(moin, rw.step, 3)
+        rtop = max(ragg.items(), key=lambda kv: kv[1]["ms"])
+        ralg = rw.algorithmic()
+        rsec = rtop[1]["ms"] * 1e-3 / rtop[1]["launches"]
+        extra["router_stress"] = {"queries_per_s": rw.Q / (rms * 1e-3), "ms_per_step": rms, "kernel": rtop[0],
+                                  "achieved_tflops": ralg["flops"] / rsec / 1e12,
+                                  "frac": ralg["flops"] / rsec / 1e12 / peaks["bf16_tflops"],
+                                  "workload": rw.config()["workload"]}
+        del rw
+        torch.cuda.empty_cache()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and kind != "forward":
+        import oracle
+        oracle.build()
+        if kind == "router":
+            n, t = adaptive_oracle(wl.oracle_sample, 64, 4096)
+            cpu = {"value": n / t, "unit": "queries/s", "cores": oracle.num_threads(), "kind": "oracle",
+                   "sample": f"{n} of {wl.Q} queries against all {wl.K} centroids, {t:.1f} s"}
+        else:
+            n, t = adaptive_oracle(wl.oracle_sample, 16, 256)
+            cpu = {"value": n / t, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
+                   "sample": f"route + 7 projections of the first {n} of {wl.T} tokens of one batch, {t:.1f} s"}
+
+    if rank == 0:
+        metric = "router_queries_per_s" if kind == "router" else "routed_lora_tokens_per_s"
+        cfg = wl.config()
+        cfg.update({"launch": "cuda_graph replay of one step" if graphed else "plain stream launches",
+                    "replicas": world, "peaks": peaks})
+        line = {"metric": metric, "value": value, "unit": wl.unit + "/s", "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": cfg, "clocks": clocks,
+                "e2e": {"value": world * wl.units_per_step / (ms_e2e * 1e-3), "unit": wl.unit + "/s",
+                        "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "ms_per_step": ms_e2e},
+                "gpu_launches": int(round(launches_per_step * args.steps)), "roofline": roof, "kernels": kernels,
+                "cpu_baseline": cpu}
+        line.update(extra)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -78,8 +78,9 @@ double moin_oracle_round_bf16(double v) { return round_bf16(v); }
  *   id[i]     = smallest k attaining max_k sim[i][k]
  *   margin[i] = best - second best (over k != id[i]); +inf when K == 1
  *
- * A zero-norm centroid has similarity -inf.  A NaN similarity never wins.  If nothing
- * wins (e.g. a zero-norm query, whose similarities are all NaN) the id is 0.
+ * A zero-norm centroid has similarity -inf, and -inf never wins.  A NaN similarity never
+ * wins.  If nothing wins (a zero-norm query, whose similarities are all NaN or -inf; or a
+ * table of zero-norm centroids) the id is 0.
  * With centroid_to_expert != NULL, expert[i] = centroid_to_expert[id[i]].
  * ------------------------------------------------------------------------------------ */
 int moin_oracle_route(const void* q, const void* c, int dtype, int64_t Q, int64_t K, int64_t D,
@@ -106,26 +107,26 @@ int moin_oracle_route(const void* q, const void* c, int dtype, int64_t Q, int64_
     double qn = sqrt(qs);
     double best = -INFINITY, second = -INFINITY;
     int64_t id = 0;
-    int have = 0;
+    int won = 0;
     for (int64_t k = 0; k < K; ++k) {
       double dot = 0.0;
       for (int64_t d = 0; d < D; ++d)
         dot += ld(q, dtype, (size_t)(i * D + d)) * ld(c, dtype, (size_t)(k * D + d));
       double sim = (cnorm[k] == 0.0) ? -INFINITY : dot / (qn * cnorm[k]);
       if (isnan(sim)) continue;
-      if (!have || sim > best) {
-        if (have) second = best;
+      if (sim > best) {          /* strict: lowest index on ties; -inf never wins */
+        second = best;
         best = sim;
         id = k;
-        have = 1;
+        won = 1;
       } else if (sim > second) {
         second = sim;
       }
     }
     if (out_centroid) out_centroid[i] = (int32_t)id;
     if (out_expert) out_expert[i] = centroid_to_expert ? centroid_to_expert[id] : (int32_t)id;
-    if (out_best) out_best[i] = have ? best : NAN;
-    if (out_margin) out_margin[i] = (K == 1 || !have) ? INFINITY : best - second;
+    if (out_best) out_best[i] = won ? best : NAN;
+    if (out_margin) out_margin[i] = (K == 1 || !won) ? INFINITY : best - second;
   }
   free(cnorm);
   return 0;

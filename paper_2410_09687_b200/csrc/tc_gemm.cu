@@ -1,10 +1,490 @@
-// placeholder until the tcgen05 kernels land: nothing is supported, callers use the warp-MMA paths
+// tcgen05 / TMEM / TMA GEMM family for sm_100a.
+//
+// One persistent, warp-specialised kernel computes D[128 x BN] tiles of  A[M,K] * B[N,K]^T
+// (both operands K-major bf16, fp32 accumulation in tensor memory):
+//   warp 0     TMA producer: 128B-swizzled [128 x 64] A boxes and [BN x 64] B boxes into a
+//              multi-stage shared-memory ring, completion on mbarriers
+//   warp 1     allocates TMEM, issues tcgen05.mma (one thread), commits stage release and
+//              accumulator-ready barriers
+//   warps 2-5  epilogue: tcgen05.ld of the accumulator (TMEM lane = tile row), then one of
+//              EPI_STORE   y = bf16(acc) (+ optional fp32 copy)
+//              EPI_ROUTER  running (max, argmax) of acc * inv_norm[col], merged across tiles with a
+//                          64-bit atomicMax on (orderable(sim) << 32 | ~col): order independent,
+//                          lowest index wins ties
+//              EPI_SHRINK  hb = bf16(scale * acc) for the LoRA rank columns
+// Two accumulator buffers in TMEM let the epilogue of tile i overlap the MMAs of tile i+1.
+//
+// Row tiles come either from a regular grid over M or from a batch plan (runs of tokens with
+// one expert, <= 128 rows).  With a plan, EPI_STORE appends one extra K block per tile taken
+// from hb[rows, r] and B_e[d_out, r] of the tile's adapter: y = [x | s h] [W ; B_e]^T, so
+// the low-rank term is added inside the accumulator and y is written once.
+// Every wait on an mbarrier is bounded; on expiry the kernel raises the status flag and returns.
+#include <cuda.h>
+
 #include "tc_gemm.cuh"
+
 namespace moin {
-bool tc_gemm_supported(int, int, int) { return false; }
-bool tc_router_supported(int, int, int) { return false; }
-bool tc_fused_supported(int) { return false; }
-moin_status launch_tc_gemm(HostState*, const __nv_bfloat16*, const __nv_bfloat16*, __nv_bfloat16*, float*, int, int, int, cudaStream_t) { return MOIN_ERR_BAD_SHAPE; }
-moin_status launch_tc_router(HostState*, const __nv_bfloat16*, const __nv_bfloat16*, const float*, int, int, int, unsigned long long*, cudaStream_t) { return MOIN_ERR_BAD_SHAPE; }
-moin_status launch_tc_lora_tiles(HostState*, const PlanView&, const moin_pool*, const __nv_bfloat16*, const __nv_bfloat16*, __nv_bfloat16*, __nv_bfloat16*, float, cudaStream_t) { return MOIN_ERR_BAD_SHAPE; }
+
+constexpr int kBM = 128, kBK = 64;
+constexpr int kTcThreads = 192;
+enum { EPI_STORE = 0, EPI_ROUTER = 1, EPI_SHRINK = 2 };
+
+struct TcParams {
+  int M, N, K;                 // problem: rows, output columns, reduction length
+  // plan tiles (nullptr -> regular grid over M)
+  const int* header;
+  const int* tile_row0;
+  const int* tile_rows;
+  const int* tile_expert;
+  const int* slot_of_expert;
+  int tail_r;                  // EPI_STORE with plan: LoRA rank of the appended K block (0 = none)
+  int rows_per_slot;           // rows of the B-side pool tensor per adapter slot (d_out, or r for EPI_SHRINK)
+  __nv_bfloat16* y;            // EPI_STORE / EPI_SHRINK output, leading dimension ldy
+  float* y0;                   // EPI_STORE: optional fp32 copy
+  int ldy;
+  float scale;                 // EPI_SHRINK
+  const float* inv_norm;       // EPI_ROUTER
+  unsigned long long* keys;    // EPI_ROUTER
+  DeviceStatus* status;
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceStatus* st,
+                                          int site) {
+  if (mbar_try_wait(bar, parity)) return true;
+  unsigned long long t0 = 0;
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 0x3FFu) == 0) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(&st->timeout_flag, 1);
+        atomicExch(&st->timeout_site, site);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
+// 8-row groups 1024 bytes apart (SBO), leading-dimension offset field 1 (unused by swizzled
+// K-major layouts), descriptor version 1, base offset 0 (tiles are 1024-byte aligned).
+__device__ __forceinline__ uint64_t make_sdesc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor: D fp32, A/B bf16, both K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t make_idesc(int bn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t orderable(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+template <int BN> struct TcCfg {
+  static constexpr int kStageBytes = (kBM + BN) * kBK * 2;
+  static constexpr int kStages = (200 * 1024) / kStageBytes > 8 ? 8 : (200 * 1024) / kStageBytes;
+  static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;   // power of two for BN in {64,128,256}
+  static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+};
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kTcThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
+  using Cfg = TcCfg<BN>;
+  constexpr int S = Cfg::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 1023u) & ~1023u;
+  uint8_t* bar_ptr = smem_raw + (tiles_base - raw) + (size_t)S * Cfg::kStageBytes;
+  const uint32_t bars = tiles_base + (uint32_t)S * Cfg::kStageBytes;
+  const uint32_t full0 = bars, empty0 = bars + 8 * S, tfull0 = bars + 16 * S, tempty0 = bars + 16 * S + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 16 * S + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + 16 * S + 40);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull0 + 8 * a, 1);
+      mbar_init(tempty0 + 8 * a, 128);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), Cfg::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const bool planned = p.header != nullptr;
+  const int tiles_n = (p.N + BN - 1) / BN;
+  const int tiles_m = planned ? p.header[PH_NTILES] : (p.M + kBM - 1) / kBM;
+  const int total = tiles_m * tiles_n;
+  const int nkb_main = (p.K + kBK - 1) / kBK;
+
+  auto tile_info = [&](int tile, int& row0, int& rows, int& n0, int& slot) {
+    const int tm = tile / tiles_n;
+    n0 = (tile - tm * tiles_n) * BN;
+    slot = -1;
+    if (planned) {
+      row0 = p.tile_row0[tm];
+      rows = p.tile_rows[tm];
+      const int e = p.tile_expert[tm];
+      if (e >= 0 && p.slot_of_expert) slot = p.slot_of_expert[e];
+    } else {
+      row0 = tm * kBM;
+      rows = min(kBM, p.M - row0);
+    }
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+        int row0, rows, n0, slot;
+        tile_info(tile, row0, rows, n0, slot);
+        const bool tail = (EPI == EPI_STORE) && planned && p.tail_r > 0 && slot >= 0;
+        const int nkb = nkb_main + (tail ? 1 : 0);
+        const int brow = (EPI == EPI_SHRINK) ? (slot >= 0 ? slot : 0) * p.rows_per_slot : n0;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const uint32_t s = it % S, ph = (it / S) & 1u;
+          if (!(ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag, p.status, 1))) break;
+          const uint32_t sa = tiles_base + s * Cfg::kStageBytes, sb = sa + kBM * kBK * 2;
+          mbar_expect_tx(full0 + 8 * s, Cfg::kStageBytes);
+          if (kb < nkb_main) {
+            tma_load_2d(sa, &tmA, full0 + 8 * s, kb * kBK, row0);
+            tma_load_2d(sb, &tmB, full0 + 8 * s, kb * kBK, brow);
+          } else {
+            tma_load_2d(sa, &tmA2, full0 + 8 * s, 0, row0);
+            tma_load_2d(sb, &tmB2, full0 + 8 * s, 0, slot * p.rows_per_slot + n0);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(BN);
+      uint32_t it = 0, lt = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++lt) {
+        int row0, rows, n0, slot;
+        tile_info(tile, row0, rows, n0, slot);
+        const bool tail = (EPI == EPI_STORE) && planned && p.tail_r > 0 && slot >= 0;
+        const int nkb = nkb_main + (tail ? 1 : 0);
+        const uint32_t acc = lt & 1u, aph = (lt >> 1) & 1u;
+        if (!(ok = mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag, p.status, 2))) break;
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + acc * BN;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const uint32_t s = it % S, ph = (it / S) & 1u;
+          if (!(ok = mbar_wait(full0 + 8 * s, ph, abort_flag, p.status, 3))) break;
+          tc_fence_after();
+          const uint32_t sa = tiles_base + s * Cfg::kStageBytes, sb = sa + kBM * kBK * 2;
+          const uint64_t da = make_sdesc(sa), db = make_sdesc(sb);
+          const int nk16 = (kb < nkb_main) ? (min(kBK, p.K - kb * kBK) + 15) / 16 : (p.tail_r + 15) / 16;
+          for (int k = 0; k < nk16; ++k)
+            tc_mma_bf16(tmem_d, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          tc_commit(empty0 + 8 * s);
+        }
+        if (ok) tc_commit(tfull0 + 8 * acc);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;             // TMEM lane quarter this warp may read
+    const int trow = q * 32 + lane;     // row of the tile owned by this thread
+    uint32_t lt = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++lt) {
+      int row0, rows, n0, slot;
+      tile_info(tile, row0, rows, n0, slot);
+      const uint32_t acc = lt & 1u, aph = (lt >> 1) & 1u;
+      if (!(ok = mbar_wait(tfull0 + 8 * acc, aph, abort_flag, p.status, 4))) break;
+      tc_fence_after();
+      const bool row_ok = trow < rows;
+      const size_t grow = (size_t)(row0 + trow);
+      float best = -INFINITY;
+      int best_k = 0;
+      const int ncols = (EPI == EPI_SHRINK) ? min(BN, (p.N + 31) / 32 * 32) : BN;
+#pragma unroll 1
+      for (int c = 0; c < ncols; c += 32) {
+        if (n0 + c >= p.N) break;
+        uint32_t v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c, v);
+        tmem_ld_wait();
+        if (EPI == EPI_ROUTER) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int k = n0 + c + j;
+            if (k < p.N) {
+              const float inv = __ldg(p.inv_norm + k);
+              const float sim = __uint_as_float(v[j]) * inv;
+              if (inv > 0.f && sim > best) {
+                best = sim;
+                best_k = k;
+              }
+            }
+          }
+        } else if (row_ok && (EPI == EPI_STORE || slot >= 0)) {
+          const float sc = (EPI == EPI_SHRINK) ? p.scale : 1.f;
+          __nv_bfloat16* yrow = p.y + grow * (size_t)p.ldy + n0 + c;
+#pragma unroll
+          for (int j = 0; j < 32; j += 8) {
+            if (n0 + c + j < p.N) {  // N is a multiple of 8
+              uint4 o;
+              o.x = pack_bf16(__uint_as_float(v[j + 0]) * sc, __uint_as_float(v[j + 1]) * sc);
+              o.y = pack_bf16(__uint_as_float(v[j + 2]) * sc, __uint_as_float(v[j + 3]) * sc);
+              o.z = pack_bf16(__uint_as_float(v[j + 4]) * sc, __uint_as_float(v[j + 5]) * sc);
+              o.w = pack_bf16(__uint_as_float(v[j + 6]) * sc, __uint_as_float(v[j + 7]) * sc);
+              *reinterpret_cast<uint4*>(yrow + j) = o;
+              if (EPI == EPI_STORE && p.y0) {
+                float* y0row = p.y0 + grow * (size_t)p.ldy + n0 + c + j;
+                *reinterpret_cast<uint4*>(y0row) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                *reinterpret_cast<uint4*>(y0row + 4) = make_uint4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(tempty0 + 8 * acc);
+      if (EPI == EPI_ROUTER && row_ok && best > -INFINITY) {
+        const unsigned long long key = ((unsigned long long)orderable(best) << 32) |
+                                       (unsigned long long)(0xFFFFFFFFu - (uint32_t)best_k);
+        atomicMax(p.keys + grow, key);
+      }
+    }
+  }
+  // ------------------------------------------------------------------ teardown
+  if (*abort_flag) {
+    // a wait ran out somewhere: give copies / MMAs still in flight time to land before the CTA's
+    // shared and tensor memory are released
+    const unsigned long long t0 = global_ns();
+    while (global_ns() - t0 < 2000000ull) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+
+static moin_status get_encoder() {
+  if (g_encode) return MOIN_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return record_cuda(e);
+  if (qres != cudaDriverEntryPointSuccess || !fn) return record_cuda(cudaErrorNotSupported);
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return MOIN_OK;
+}
+
+// 2-D row-major bf16 tensor [rows, cols] -> map with a [box_rows x 64] box, 128-byte swizzle, zero fill.
+static moin_status make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  moin_status st = get_encoder();
+  if (st) return st;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return record_cuda(cudaErrorInvalidValue);
+  return MOIN_OK;
+}
+
+template <int BN, int EPI>
+static moin_status launch_cfg(HostState* hs, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& a2,
+                              const CUtensorMap& b2, const TcParams& p, long max_tiles, cudaStream_t stream) {
+  using Cfg = TcCfg<BN>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)Cfg::kSmemBytes);
+    if (e != cudaSuccess) return record_cuda(e);
+    configured = true;
+  }
+  long grid = max_tiles < hs->n_sms ? max_tiles : hs->n_sms;
+  if (grid < 1) grid = 1;
+  tc_gemm_kernel<BN, EPI><<<(int)grid, kTcThreads, Cfg::kSmemBytes, stream>>>(a, b, a2, b2, p);
+  return record_cuda(cudaGetLastError());
+}
+
+static int pick_bn(long tiles_m, int N, int n_sms) {
+  for (int bn : {256, 128}) {
+    if (tiles_m * ((N + bn - 1) / bn) >= n_sms) return bn;
+  }
+  return 64;
+}
+
+bool tc_gemm_supported(int T, int d_in, int d_out) { return T >= 1 && d_in >= 64 && (d_in % 8) == 0 && (d_out % 8) == 0; }
+bool tc_router_supported(int Q, int K, int D) { return Q >= 1 && K >= 1 && D >= 64 && (D % 8) == 0; }
+bool tc_fused_supported(int r) { return r >= 8 && r <= 64 && (r % 8) == 0; }
+
+moin_status launch_tc_gemm(HostState* hs, const __nv_bfloat16* x, const __nv_bfloat16* W, __nv_bfloat16* y, float* y0,
+                           int T, int d_in, int d_out, cudaStream_t stream) {
+  const long tiles_m = (T + kBM - 1) / kBM;
+  const int bn = pick_bn(tiles_m, d_out, hs->n_sms);
+  CUtensorMap a, b;
+  moin_status st = make_map(&a, x, T, d_in, kBM);
+  if (!st) st = make_map(&b, W, d_out, d_in, bn);
+  if (st) return st;
+  TcParams p = {};
+  p.M = T; p.N = d_out; p.K = d_in; p.y = y; p.y0 = y0; p.ldy = d_out; p.scale = 1.f; p.status = hs->status;
+  const long tiles = tiles_m * ((d_out + bn - 1) / bn);
+  if (bn == 256) return launch_cfg<256, EPI_STORE>(hs, a, b, a, b, p, tiles, stream);
+  if (bn == 128) return launch_cfg<128, EPI_STORE>(hs, a, b, a, b, p, tiles, stream);
+  return launch_cfg<64, EPI_STORE>(hs, a, b, a, b, p, tiles, stream);
+}
+
+moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
+                             int Q, int K, int D, unsigned long long* keys, cudaStream_t stream) {
+  const long tiles_m = (Q + kBM - 1) / kBM;
+  const int bn = pick_bn(tiles_m, K, hs->n_sms);
+  CUtensorMap a, b;
+  moin_status st = make_map(&a, q, Q, D, kBM);
+  if (!st) st = make_map(&b, c, K, D, bn);
+  if (st) return st;
+  TcParams p = {};
+  p.M = Q; p.N = K; p.K = D; p.inv_norm = inv_norm; p.keys = keys; p.status = hs->status;
+  const long tiles = tiles_m * ((K + bn - 1) / bn);
+  if (bn == 256) return launch_cfg<256, EPI_ROUTER>(hs, a, b, a, b, p, tiles, stream);
+  if (bn == 128) return launch_cfg<128, EPI_ROUTER>(hs, a, b, a, b, p, tiles, stream);
+  return launch_cfg<64, EPI_ROUTER>(hs, a, b, a, b, p, tiles, stream);
+}
+
+moin_status launch_tc_lora_tiles(HostState* hs, const PlanView& pv, const moin_pool* pool, const __nv_bfloat16* x,
+                                 const __nv_bfloat16* W, __nv_bfloat16* y, __nv_bfloat16* hb, float scale,
+                                 cudaStream_t stream) {
+  const int T = pv.T, d_in = pool->d_in, d_out = pool->d_out, r = pool->r;
+  // upper bound on row tiles without reading the plan back: every run adds at most one partial tile
+  const long max_tiles_m = T;  // grid is capped at the SM count; the kernel reads the true count
+  CUtensorMap ax, bA, bW, ah, bB;
+  moin_status st = make_map(&ax, x, T, d_in, kBM);
+  if (!st) st = make_map(&bA, pool->A, (uint64_t)pool->n_slots * r, d_in, 64);
+  if (!st) st = make_map(&ah, hb, T, r, kBM);
+  if (!st) st = make_map(&bB, pool->B, (uint64_t)pool->n_slots * d_out, r, 256);
+  if (st) return st;
+  // 1. hb[row, :r] = bf16(scale * x A_e^T)   (one N tile of 64 columns, rank columns stored)
+  {
+    ProfScope prof(MOIN_K_SHRINK_TC, 1, stream);
+    TcParams p = {};
+    p.M = T; p.N = r; p.K = d_in; p.header = pv.header; p.tile_row0 = pv.tile_row0; p.tile_rows = pv.tile_rows;
+    p.tile_expert = pv.tile_expert; p.slot_of_expert = pool->slot_of_expert; p.rows_per_slot = r; p.y = hb; p.ldy = r;
+    p.scale = scale; p.status = hs->status;
+    st = launch_cfg<64, EPI_SHRINK>(hs, ax, bA, ax, bA, p, max_tiles_m, stream);
+    if (st) return st;
+  }
+  // 2. y = [x | hb] [W ; B_e]^T
+  ProfScope prof(MOIN_K_FUSED_TC, 1, stream);
+  const long full_tiles_m = (T + kBM - 1) / kBM;
+  const int bn = pick_bn(full_tiles_m, d_out, hs->n_sms);
+  st = make_map(&bW, W, d_out, d_in, bn);
+  if (!st && bn != 256) st = make_map(&bB, pool->B, (uint64_t)pool->n_slots * d_out, r, bn);
+  if (st) return st;
+  TcParams p = {};
+  p.M = T; p.N = d_out; p.K = d_in; p.header = pv.header; p.tile_row0 = pv.tile_row0; p.tile_rows = pv.tile_rows;
+  p.tile_expert = pv.tile_expert; p.slot_of_expert = pool->slot_of_expert; p.tail_r = r; p.rows_per_slot = d_out;
+  p.y = y; p.ldy = d_out; p.scale = 1.f; p.status = hs->status;
+  const long tiles = max_tiles_m * ((d_out + bn - 1) / bn);
+  if (bn == 256) return launch_cfg<256, EPI_STORE>(hs, ax, bW, ah, bB, p, tiles, stream);
+  if (bn == 128) return launch_cfg<128, EPI_STORE>(hs, ax, bW, ah, bB, p, tiles, stream);
+  return launch_cfg<64, EPI_STORE>(hs, ax, bW, ah, bB, p, tiles, stream);
+}
+
+}  // namespace moin

@@ -90,6 +90,11 @@ def test_degenerate_vectors():
     assert out["centroid"][0] == 1           # zero-norm centroid never chosen
     assert out["centroid"][1] == 0           # zero-norm query: id 0
     assert out["centroid"][2] == 1           # ties at -0.707: lowest valid index
+    # the zero-norm centroid is not first: a zero-norm query still gets id 0 (nothing wins), not 1
+    c2 = np.array([[1.0, 0.0], [0.0, 0.0], [0.0, 1.0]])
+    out2 = oracle.route(np.array([[0.0, 0.0], [0.2, 1.0]]), c2)
+    assert out2["centroid"][0] == 0 and np.isnan(out2["best"][0]) and out2["centroid"][1] == 2
+    assert oracle.route(np.array([[1.0, 1.0]]), np.zeros((3, 2)))["centroid"][0] == 0   # all centroids zero
     one = oracle.route(np.array([[1.0, 2.0]]), np.array([[3.0, 1.0]]))
     assert one["centroid"][0] == 0 and np.isinf(one["margin"][0])
 
