@@ -30,6 +30,12 @@ moin_status host_state(HostState** out) {
     e = cudaGetSymbolAddress(&p, g_device_status);
     if (e != cudaSuccess) return record_cuda(e);
     g_state.status = reinterpret_cast<DeviceStatus*>(p);
+    if (g_state.side == nullptr) {
+      e = cudaStreamCreateWithFlags(&g_state.side, cudaStreamNonBlocking);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_state.ev_fork, cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_state.ev_join, cudaEventDisableTiming);
+      if (e != cudaSuccess) return record_cuda(e);
+    }
     g_state.n_sms = prop.multiProcessorCount;
     g_state.device = dev;
   }
@@ -346,23 +352,32 @@ moin_status moin_lora_linear(const moin_plan* plan, const void* x, const void* W
     __nv_bfloat16* hb = reinterpret_cast<__nv_bfloat16*>(ws);  // [T, r] bf16, s * (x A^T)
     return launch_tc_lora_tiles(hs, pv, pool, xb, Wb, yb, hb, scale, s);
   }
-  // Short segments: base GEMM (y and fp32 y0), then stream every distinct adapter once.
+  // Short segments: the base GEMM (y and fp32 y0) and the shrink are independent, so the GEMM runs on
+  // the library's side stream between a fork and a join event; the expand then adds y0 + s h B^T.
   float* h = reinterpret_cast<float*>(ws);
   float* y0 = reinterpret_cast<float*>(ws + align_up((size_t)T * (size_t)r * sizeof(float), 256));
+  cudaError_t ce = cudaEventRecord(hs->ev_fork, s);
+  if (ce == cudaSuccess) ce = cudaStreamWaitEvent(hs->side, hs->ev_fork, 0);
+  if (ce != cudaSuccess) return record_cuda(ce);
   {
-    ProfScope prof(use_tc ? MOIN_K_GEMM_TC : MOIN_K_GEMM_WARP, 1, s);
+    ProfScope prof(use_tc ? MOIN_K_GEMM_TC : MOIN_K_GEMM_WARP, 1, hs->side);
     if (use_tc)
-      st = launch_tc_gemm(hs, xb, Wb, yb, y0, T, d_in, d_out, s);
+      st = launch_tc_gemm(hs, xb, Wb, yb, y0, T, d_in, d_out, hs->side);
     else
-      st = record_cuda(launch_gemm_warp(xb, Wb, yb, y0, T, d_in, d_out, s));
+      st = record_cuda(launch_gemm_warp(xb, Wb, yb, y0, T, d_in, d_out, hs->side));
   }
-  if (st) return st;
+  moin_status st2;
   {
     ProfScope prof(MOIN_K_SHRINK_STREAM, 1, s);
-    st = record_cuda(launch_lora_shrink_stream(pv, pool->slot_of_expert, xb, (const __nv_bfloat16*)pool->A, h, r, d_in,
-                                               hs->n_sms, s));
+    st2 = record_cuda(launch_lora_shrink_stream(pv, pool->slot_of_expert, xb, (const __nv_bfloat16*)pool->A, h, r, d_in,
+                                                hs->n_sms, s));
   }
+  // always join, even after a failed launch, so the side stream never outlives the call's ordering
+  ce = cudaEventRecord(hs->ev_join, hs->side);
+  if (ce == cudaSuccess) ce = cudaStreamWaitEvent(s, hs->ev_join, 0);
   if (st) return st;
+  if (st2) return st2;
+  if (ce != cudaSuccess) return record_cuda(ce);
   ProfScope prof(MOIN_K_EXPAND_STREAM, 1, s);
   return record_cuda(launch_lora_expand_stream(pv, pool->slot_of_expert, h, (const __nv_bfloat16*)pool->B, y0, yb,
                                                scale, r, d_out, hs->n_sms, s));

@@ -128,6 +128,9 @@ struct HostState {
   int device = -1;
   int n_sms = 0;
   int gemm_impl = 0;               // MOIN_OPT_GEMM_IMPL
+  // fork/join inside one call: independent kernels of a call run on `side` between two events
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 moin_status host_state(HostState** out);      // lazily initialised for the current device
 moin_status record_cuda(cudaError_t e);       // MOIN_OK or MOIN_ERR_CUDA (remembers e)
