@@ -129,6 +129,25 @@ moin_status moin_route(const moin_router* router, const void* queries, int32_t Q
                        int32_t* out_centroid, float* out_best_sim, void* workspace, size_t workspace_bytes,
                        moin_stream stream);
 
+/* Routing for callers that cannot hand the library a workspace.  (The paper has no counterpart: this is
+ * a packaging variant of moin_route, added for processes that must not allocate device memory - e.g. a
+ * serving worker whose memory pool was sized and frozen at start-up, or a plug-in that runs inside
+ * someone else's CUDA context and is forbidden to call cudaMalloc.)
+ *
+ * It computes exactly what moin_route computes, with the same arguments minus the workspace.  The
+ * per-query scratch that the tensor-core router needs lives in a fixed array inside the library image
+ * (MOIN_ROUTE_STATIC_MAX_Q * 8 bytes = 512 KiB, held by every GPU that loads the library until the
+ * process exits).  The call performs no cudaMalloc/cudaFree and calls no allocating routine.
+ *   - Q > MOIN_ROUTE_STATIC_MAX_Q returns MOIN_ERR_WORKSPACE and launches nothing.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents; the part a call uses is
+ *     cleared on `stream` before use.  Two calls whose GPU work overlaps (different streams, no ordering
+ *     between them) race on it: order them, or use moin_route with separate workspaces. */
+enum { MOIN_ROUTE_STATIC_MAX_Q = 65536 };
+moin_status moin_route_static(const moin_router* router, const void* queries, int32_t Q, int32_t* out_expert,
+                              int32_t* out_centroid, float* out_best_sim, moin_stream stream);
+
 /* ---------------------------------------------------------------------------------------
  * Adapter pool of ONE projection.  Paper Sec. 3.2: W_a in R^{r x d}, W_b in R^{k x r} per
  * expert and linear layer; Sec. 1: the adapters in use are kept in GPU memory.  The pool

@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = (
     "moin_set_option", "moin_router_prepare", "moin_route_workspace_bytes", "moin_route", "moin_plan_bytes",
     "moin_plan_build", "moin_plan_read", "moin_lora_linear_workspace_bytes", "moin_lora_linear",
     "moin_decoder_workspace_bytes", "moin_decoder_forward", "moin_profile_enable", "moin_profile_read",
-    "moin_kernel_name",
+    "moin_kernel_name", "moin_route_static",
 )
 
 
@@ -92,6 +92,7 @@ def lib() -> ctypes.CDLL:
         L.moin_route_workspace_bytes.restype = sz
         L.moin_route_workspace_bytes.argtypes = [i32, i32, i32]
         L.moin_route.argtypes = [ctypes.POINTER(_Router), vp, i32, vp, vp, vp, vp, sz, vp]
+        L.moin_route_static.argtypes = [ctypes.POINTER(_Router), vp, i32, vp, vp, vp, vp]
         L.moin_plan_bytes.restype = sz
         L.moin_plan_bytes.argtypes = [i32, i32]
         L.moin_plan_build.argtypes = [vp, ctypes.POINTER(_Plan), vp]
@@ -198,6 +199,23 @@ def route(router: Router, queries: torch.Tensor, out_expert: Optional[torch.Tens
     ws = router.workspace(Q)
     _check(lib().moin_route(ctypes.byref(router.c), _ptr(queries), Q, _ptr(out_expert), _ptr(out_centroid),
                             _ptr(out_best_sim), _ptr(ws), ws.numel(), _stream(stream)), "moin_route")
+    return out_expert
+
+
+ROUTE_STATIC_MAX_Q = 65536
+
+
+def route_static(router: Router, queries: torch.Tensor, out_expert: torch.Tensor,
+                 out_centroid: Optional[torch.Tensor] = None, out_best_sim: Optional[torch.Tensor] = None,
+                 stream=None) -> torch.Tensor:
+    """moin_route_static: the router for callers that may not allocate device memory.
+
+    Same result as ``route``; the scratch lives inside the library (at most ROUTE_STATIC_MAX_Q queries per
+    call).  This wrapper allocates nothing either: the caller passes every output tensor.  Calls share
+    the built-in scratch, so calls that overlap on the GPU race - keep them ordered on one stream."""
+    assert queries.dtype == torch.bfloat16 and queries.dim() == 2 and queries.shape[1] == router.D
+    _check(lib().moin_route_static(ctypes.byref(router.c), _ptr(queries), queries.shape[0], _ptr(out_expert),
+                                   _ptr(out_centroid), _ptr(out_best_sim), _stream(stream)), "moin_route_static")
     return out_expert
 
 

@@ -222,6 +222,53 @@ moin_status moin_route(const moin_router* router, const void* queries, int32_t Q
                                          out_centroid, out_best_sim, s));
 }
 
+/* Scratch of moin_route_static: one 64-bit (similarity, index) key per query.  In host code the name
+ * `g_route_static_keys` is only a handle for the runtime, not a device address; the address handed to
+ * kernels comes from cudaGetSymbolAddress, looked up once per device. */
+static __device__ __align__(256) unsigned long long g_route_static_keys[MOIN_ROUTE_STATIC_MAX_Q];
+static unsigned long long* g_route_static_ptr[64] = {nullptr};
+
+moin_status moin_route_static(const moin_router* router, const void* queries, int32_t Q, int32_t* out_expert,
+                              int32_t* out_centroid, float* out_best_sim, moin_stream stream) {
+  if (!router || Q < 0) return MOIN_ERR_INVALID_ARG;
+  if (Q == 0) return MOIN_OK;
+  if (Q > MOIN_ROUTE_STATIC_MAX_Q) return MOIN_ERR_WORKSPACE;   // beyond the built-in scratch
+  if (!queries || !out_expert || !router->centroids || !router->inv_norm || router->K < 1) return MOIN_ERR_INVALID_ARG;
+  const int K = router->K, D = router->D;
+  if (D < 8 || D > 8192 || (D % 8) != 0) return MOIN_ERR_BAD_SHAPE;
+  if (!aligned16(queries) || !aligned16(router->centroids)) return MOIN_ERR_MISALIGNED;
+  HostState* hs;
+  moin_status st = host_state(&hs);
+  if (st) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (!tc_router_supported(Q, K, D)) {   // tiny embedding dimension: the CUDA-core kernel needs no scratch
+    ProfScope prof(MOIN_K_ROUTE_SIMPLE, 1, s);
+    return record_cuda(launch_route_simple((const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids,
+                                           router->inv_norm, router->centroid_to_expert, Q, K, D, out_expert,
+                                           out_centroid, out_best_sim, s));
+  }
+  if (hs->device < 0 || hs->device >= 64) return MOIN_ERR_NO_DEVICE;
+  if (g_route_static_ptr[hs->device] == nullptr) {   // set-up: once per device, that device is current here
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_route_static_keys);
+    if (e != cudaSuccess) return record_cuda(e);
+    g_route_static_ptr[hs->device] = reinterpret_cast<unsigned long long*>(p);
+  }
+  unsigned long long* keys = g_route_static_ptr[hs->device];
+  // the array still holds the previous call's keys: the merge is a max, so it must start from zero
+  cudaError_t e = cudaMemsetAsync(keys, 0, (size_t)Q * sizeof(unsigned long long), s);
+  if (e != cudaSuccess) return record_cuda(e);
+  {
+    ProfScope prof(MOIN_K_ROUTE_TC, 1, s);
+    st = launch_tc_router(hs, (const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids,
+                          router->inv_norm, Q, K, D, keys, s);
+  }
+  if (st) return st;
+  ProfScope prof(MOIN_K_ROUTE_FINISH, 1, s);
+  return record_cuda(launch_route_finish(keys, (const __nv_bfloat16*)queries, router->centroid_to_expert, Q, D,
+                                         out_expert, out_centroid, out_best_sim, s));
+}
+
 /* ------------------------------------------------------------------ plan */
 
 size_t moin_plan_bytes(int32_t T, int32_t E) {
