@@ -420,7 +420,7 @@ def profile_pass(moin, fn, steps: int):
 
 def traffic_for(kernel: str, workload: str):
     """DRAM bytes per launch from the committed ncu capture, or None when the kernel source changed since."""
-    p = os.path.join(ROOT, "profiles", "traffic.json")
+    p = os.path.join(ROOT, "profiles", "dram_traffic.txt")
     if not os.path.exists(p):
         return None
     try:
