@@ -289,7 +289,7 @@ moin_status moin_plan_build(const int32_t* token_expert, moin_plan* plan, moin_s
   cudaStream_t s = (cudaStream_t)stream;
   PlanView v = plan_view(plan->buffer, plan->T, plan->E);
   {
-    ProfScope prof(MOIN_K_PLAN, 3, s);
+    ProfScope prof(MOIN_K_PLAN, plan->T > kPlanChunk ? 4 : 3, s);
     st = record_cuda(launch_plan_build(token_expert, v, hs->status, s));
   }
   if (st) return st;

@@ -1,8 +1,9 @@
 // Batch plan: grouping of tokens by expert id (integer work only).
 //
-// Three small launches:
+// A few small launches:
 //   plan_rank_kernel    per 256-token chunk: sanitise ids, stable in-chunk rank, per-chunk histogram
-//   plan_scan_kernel    one CTA: prefix over chunks and over expert ids -> segment list; run tiles
+//   plan_prefix_kernel  (batches of more than one chunk) per expert id: prefix of its counts over the chunks
+//   plan_scan_kernel    one CTA: prefix over expert ids -> segment list; run tiles
 //   plan_scatter_kernel per chunk: position = expert base + chunk prefix + in-chunk rank -> perm
 // The result is a stable counting sort (token order is kept inside every expert segment), so
 // the plan is deterministic.
@@ -92,15 +93,35 @@ __device__ __forceinline__ int block_incl_max_1024(int v, int* smem) {
   return max(inc, prev);
 }
 
-__global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v) {
+// Per expert id: exclusive prefix of its per-chunk counts over the chunks (in place) and the total.
+// One thread per expert id; counts are read in batches so the loads of a batch are in flight together.
+__global__ void __launch_bounds__(256) plan_prefix_kernel(PlanView v) {
+  const int k = blockIdx.x * 256 + threadIdx.x;
+  if (k > v.E) return;
+  const size_t pitch = (size_t)(v.E + 1);
+  int run = 0;
+  for (int c0 = 0; c0 < v.n_chunks; c0 += 8) {
+    int n[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) n[j] = (c0 + j < v.n_chunks) ? __ldcg(v.hist + (size_t)(c0 + j) * pitch + k) : 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (c0 + j < v.n_chunks) v.hist[(size_t)(c0 + j) * pitch + k] = run;
+      run += n[j];
+    }
+  }
+  v.keybase[k] = run;
+}
+
+__global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_prefix) {
   __shared__ int smem[33];
   __shared__ int s_carry[2];
   const int tid = threadIdx.x;
   const int T = v.T, E = v.E, nc = v.n_chunks;
   const size_t pitch = (size_t)(E + 1);
 
-  // 1. per expert id: prefix over chunks (in place) and total
-  for (int k = tid; k <= E; k += 1024) {
+  // 1. per expert id: prefix over chunks (in place) and total (done by plan_prefix_kernel for multi-chunk batches)
+  for (int k = tid; do_prefix && k <= E; k += 1024) {
     int run = 0;
     for (int c = 0; c < nc; ++c) {
       int* p = v.hist + (size_t)c * pitch + k;
@@ -183,7 +204,8 @@ cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, Device
   cudaError_t e = cudaMemsetAsync(v.hist, 0, sizeof(int) * (size_t)v.n_chunks * (size_t)(v.E + 1), stream);
   if (e != cudaSuccess) return e;
   plan_rank_kernel<<<v.n_chunks, kPlanChunk, 0, stream>>>(token_expert, v.T, v.E, v.key, v.rank, v.hist, status);
-  plan_scan_kernel<<<1, 1024, 0, stream>>>(v);
+  if (v.n_chunks > 1) plan_prefix_kernel<<<(v.E + 1 + 255) / 256, 256, 0, stream>>>(v);
+  plan_scan_kernel<<<1, 1024, 0, stream>>>(v, v.n_chunks > 1 ? 0 : 1);
   plan_scatter_kernel<<<v.n_chunks, kPlanChunk, 0, stream>>>(v);
   return cudaGetLastError();
 }
