@@ -30,6 +30,7 @@ struct PlanView {   // pointers into the plan buffer
   int* perm;         // [T]   token indices ordered by (expert, token)
   int* seg_expert;   // [Smax]
   int* seg_start;    // [Smax + 1]
+  int4* seg_tab;     // [Smax + 1] packed (expert, start, length, 0): one 16-byte load per segment
   int* tile_row0;    // [T + 1]
   int* tile_rows;    // [T]
   int* tile_expert;  // [T]
@@ -54,6 +55,7 @@ inline PlanView plan_view(void* buffer, int T, int E, size_t* total_words = null
   v.perm = take(T);
   v.seg_expert = take(v.Smax + 1);
   v.seg_start = take(v.Smax + 2);
+  v.seg_tab = reinterpret_cast<int4*>(take(4 * (size_t)(v.Smax + 1)));
   v.tile_row0 = take(T + 1);
   v.tile_rows = take(T + 1);
   v.tile_expert = take(T + 1);

@@ -146,6 +146,7 @@ __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_pref
       if (n > 0) {
         v.seg_expert[carry_seg + ex_seg] = k;
         v.seg_start[carry_seg + ex_seg] = carry_tok + ex_tok;
+        v.seg_tab[carry_seg + ex_seg] = make_int4(k, carry_tok + ex_tok, n, 0);
       }
     }
     max_seg = max(max_seg, n);

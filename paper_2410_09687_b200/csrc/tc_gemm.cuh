@@ -1,8 +1,14 @@
 // tcgen05 / TMEM / TMA GEMM family (host-side interface).
 #pragma once
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace moin {
+
+// 2-D row-major bf16 tensor [rows, cols] -> TMA map with a [box_rows x 64] box, 128-byte swizzle, zero fill
+// (columns of the box beyond `cols` read as zero).
+moin_status make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 
 // Shape predicates (host): can the tcgen05 kernels take this problem?
 bool tc_gemm_supported(int T, int d_in, int d_out);
@@ -19,5 +25,14 @@ moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_b
 moin_status launch_tc_lora_tiles(HostState* hs, const PlanView& pv, const moin_pool* pool, const __nv_bfloat16* x,
                                  const __nv_bfloat16* W, __nv_bfloat16* y, __nv_bfloat16* hb, float scale,
                                  cudaStream_t stream);
+
+// TMA-staged segmented LoRA kernels (short segments).  The shrink writes lora_stream_parts(d_in) partial
+// results hpart[part][T][r]; the expand sums them in a fixed order.
+int lora_stream_parts(int d_in);
+bool lora_shrink_tma_supported(int d_in);
+moin_status launch_lora_shrink_tma(HostState* hs, const PlanView& pv, const moin_pool* pool, const __nv_bfloat16* x,
+                                   float* hpart, cudaStream_t stream);
+moin_status launch_lora_expand_tma(HostState* hs, const PlanView& pv, const moin_pool* pool, const float* hpart, int KP,
+                                   const float* y0, __nv_bfloat16* y, float scale, cudaStream_t stream);
 
 }  // namespace moin
