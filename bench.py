@@ -514,6 +514,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-router-extra", action="store_true")
     ap.add_argument("--forward-layers", type=int, default=22)
+    ap.add_argument("--stream-impl", type=int, default=0, help="short-segment LoRA kernels: 0 auto, 1 register-fed, 2 TMA-staged")
     args = ap.parse_args()
     defaults = {"decode": (3000, 20), "prefill": (100, 5), "router": (50, 5), "forward": (5, 3)}
     if args.impl == "reference":
@@ -530,6 +531,7 @@ def main():
         from paper_2410_09687_b200 import build
         build.build()
     moin.lib()
+    moin.set_option(moin.OPT_STREAM_IMPL, args.stream_impl)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
     world, rank, local = dist_setup(args.gpus)

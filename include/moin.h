@@ -76,7 +76,8 @@ moin_status moin_device_status_reset(moin_stream stream);
 /* Testing/tuning knobs (host-side path selection only; every path computes the same function).
  *   MOIN_OPT_GEMM_IMPL: 0 = automatic, 1 = force the warp-MMA kernels, 2 = force the tcgen05 kernels
  *                       (calls whose shapes the forced kernel cannot take fail with MOIN_ERR_BAD_SHAPE). */
-enum { MOIN_OPT_GEMM_IMPL = 1 };
+/*   MOIN_OPT_STREAM_IMPL: short-segment LoRA kernels: 0 = automatic, 1 = register-fed kernels, 2 = TMA-staged kernels. */
+enum { MOIN_OPT_GEMM_IMPL = 1, MOIN_OPT_STREAM_IMPL = 2 };
 moin_status moin_set_option(int32_t key, int32_t value);
 
 /* Per-kernel timing for benchmarks (no counterpart in the paper).  While enabled, every kernel group the

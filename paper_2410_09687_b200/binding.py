@@ -15,6 +15,7 @@ _lib: Optional[ctypes.CDLL] = None
 PLAN_AUTO, PLAN_SEGMENTS, PLAN_TILES = 0, 1, 2
 LOGITS_ALL, LOGITS_LAST, LOGITS_NONE = 0, 1, 2
 OPT_GEMM_IMPL = 1
+OPT_STREAM_IMPL = 2
 
 EXPORTED_SYMBOLS = (
     "moin_status_string", "moin_version", "moin_last_cuda_error", "moin_device_status", "moin_device_status_reset",

@@ -96,6 +96,10 @@ moin_status moin_set_option(int32_t key, int32_t value) {
     g_state.gemm_impl = value;
     return MOIN_OK;
   }
+  if (key == MOIN_OPT_STREAM_IMPL && value >= 0 && value <= 2) {
+    g_state.stream_impl = value;
+    return MOIN_OK;
+  }
   return MOIN_ERR_INVALID_ARG;
 }
 
@@ -339,10 +343,10 @@ moin_status moin_plan_read(const moin_plan* plan, int32_t* n_segments, int32_t* 
 /* ------------------------------------------------------------------ routed LoRA linear layer */
 
 size_t moin_lora_linear_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, int32_t r) {
-  (void)d_in;
   if (T <= 0) return 256;
   const size_t Tp = align_up((size_t)T, kTileRows) + kTileRows;
-  size_t seg = align_up((size_t)T * (size_t)(r > 0 ? r : 8) * sizeof(float), 256) +
+  const size_t parts = (size_t)lora_stream_parts(d_in > 0 ? d_in : 64);
+  size_t seg = align_up(parts * (size_t)T * (size_t)(r > 0 ? r : 8) * sizeof(float), 256) +
                align_up((size_t)T * (size_t)d_out * sizeof(float), 256);
   size_t tiles = align_up(Tp * (size_t)64 * sizeof(__nv_bfloat16), 256);
   return (seg > tiles ? seg : tiles) + 256;
@@ -401,8 +405,11 @@ moin_status moin_lora_linear(const moin_plan* plan, const void* x, const void* W
   }
   // Short segments: the base GEMM (y and fp32 y0) and the shrink are independent, so the GEMM runs on
   // the library's side stream between a fork and a join event; the expand then adds y0 + s h B^T.
-  float* h = reinterpret_cast<float*>(ws);
-  float* y0 = reinterpret_cast<float*>(ws + align_up((size_t)T * (size_t)r * sizeof(float), 256));
+  const bool tma_stream = hs->stream_impl != 1;                 // MOIN_OPT_STREAM_IMPL
+  const bool tma_shrink = tma_stream && lora_shrink_tma_supported(d_in);
+  const int parts = tma_shrink ? lora_stream_parts(d_in) : 1;
+  float* h = reinterpret_cast<float*>(ws);                      // [parts][T][r] partial shrink results
+  float* y0 = reinterpret_cast<float*>(ws + align_up((size_t)lora_stream_parts(d_in) * (size_t)T * (size_t)r * sizeof(float), 256));
   cudaError_t ce = cudaEventRecord(hs->ev_fork, s);
   if (ce == cudaSuccess) ce = cudaStreamWaitEvent(hs->side, hs->ev_fork, 0);
   if (ce != cudaSuccess) return record_cuda(ce);
@@ -416,8 +423,11 @@ moin_status moin_lora_linear(const moin_plan* plan, const void* x, const void* W
   moin_status st2;
   {
     ProfScope prof(MOIN_K_SHRINK_STREAM, 1, s);
-    st2 = record_cuda(launch_lora_shrink_stream(pv, pool->slot_of_expert, xb, (const __nv_bfloat16*)pool->A, h, r, d_in,
-                                                hs->n_sms, s));
+    if (tma_shrink)
+      st2 = launch_lora_shrink_tma(hs, pv, pool, xb, h, s);
+    else
+      st2 = record_cuda(launch_lora_shrink_stream(pv, pool->slot_of_expert, xb, (const __nv_bfloat16*)pool->A, h, r,
+                                                  d_in, hs->n_sms, s));
   }
   // always join, even after a failed launch, so the side stream never outlives the call's ordering
   ce = cudaEventRecord(hs->ev_join, hs->side);
@@ -426,6 +436,7 @@ moin_status moin_lora_linear(const moin_plan* plan, const void* x, const void* W
   if (st2) return st2;
   if (ce != cudaSuccess) return record_cuda(ce);
   ProfScope prof(MOIN_K_EXPAND_STREAM, 1, s);
+  if (tma_stream) return launch_lora_expand_tma(hs, pv, pool, h, parts, y0, yb, scale, s);
   return record_cuda(launch_lora_expand_stream(pv, pool->slot_of_expert, h, (const __nv_bfloat16*)pool->B, y0, yb,
                                                scale, r, d_out, hs->n_sms, s));
 }

@@ -130,6 +130,7 @@ struct HostState {
   int device = -1;
   int n_sms = 0;
   int gemm_impl = 0;               // MOIN_OPT_GEMM_IMPL
+  int stream_impl = 0;             // MOIN_OPT_STREAM_IMPL
   // fork/join inside one call: independent kernels of a call run on `side` between two events
   cudaStream_t side = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;

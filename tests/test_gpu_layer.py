@@ -37,11 +37,20 @@ def test_tiny_config_routed_by_the_router():
     assert_layer_close(y, oracle_layer(case), "tiny routed")
 
 
+@pytest.fixture(params=[1, 2], ids=["regfed", "tma"])
+def stream_impl(request):
+    """Both implementations of the short-segment kernels (register-fed and TMA-staged)."""
+    moin.set_option(moin.OPT_STREAM_IMPL, request.param)
+    yield request.param
+    moin.set_option(moin.OPT_STREAM_IMPL, 0)
+
+
 @pytest.mark.parametrize("r", [8, 16, 24, 32, 40, 48, 56, 64])
 @pytest.mark.parametrize("mode", MODES)
-def test_every_supported_rank(r, mode):
+def test_every_supported_rank(r, mode, stream_impl):
     rng = mi.np_rng(7, r)
-    E, T, d_in, d_out = 6, 333, 192, 328     # ragged T, d_out not a multiple of 16 or 64
+    # ragged T, d_out not a multiple of 16 or 64; d_in alternates between a multiple of 256 and not
+    E, T, d_in, d_out = 6, 333, (192 if r % 16 else 512), 328
     pool = mi.make_pool(E, r, d_in, d_out, 7, r, missing=(4,))
     lens = rng.multinomial(T - 8, [1 / 8] * 8) + 1
     te = np.repeat(rng.integers(-1, E, size=8), lens).astype(np.int32)
@@ -51,7 +60,7 @@ def test_every_supported_rank(r, mode):
 
 
 @pytest.mark.parametrize("mode", MODES)
-def test_base_only_and_missing_adapters(mode):
+def test_base_only_and_missing_adapters(mode, stream_impl):
     pool = mi.make_pool(5, 16, 256, 128, 8, 1, missing=(1, 3))
     te = np.array([-1, 1, 3, 0, 2, 4, 99, -5] * 20, np.int32)
     case = mi.layer_case("fallback", len(te), 256, 128, pool, te, 2.0, 8, 2)
@@ -67,7 +76,7 @@ def test_base_only_and_missing_adapters(mode):
                                                   None, 0.0), "base")
 
 
-def test_decode_config_all_projections():
+def test_decode_config_all_projections(stream_impl):
     # 256 single-token requests, 500 rank-64 experts: every token checked against the oracle.
     cases = mi.decode_batch(seed=1, device=DEV)
     te = cases[0].token_expert
@@ -94,7 +103,7 @@ def test_prefill_config_sampled_rows():
 
 
 @pytest.mark.parametrize("mode", MODES)
-def test_request_permutation_and_determinism(mode):
+def test_request_permutation_and_determinism(mode, stream_impl):
     # experts do not interact: permuting requests permutes output rows (bitwise), and reruns are bitwise equal
     pool = mi.make_pool(12, 32, 256, 256, 9, 1)
     rng = mi.np_rng(9, 2)
