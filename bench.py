@@ -38,6 +38,7 @@ import moin_inputs as mi
 NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 ROTATE = 4  # distinct input batches rotated through the timed steps
+GROUPS = [[0, 1, 2], [3], [4, 5], [6]]  # {q,k,v}, {o}, {gate,up}, {down}: independent inside a decoder block
 
 
 def load_peaks():
@@ -107,9 +108,9 @@ class ClockSampler:
 class LayerWorkload:
     """route -> plan -> seven projections.  decode: E=500 r=64 T=256; prefill: E=5000 r=16 32x512."""
 
-    def __init__(self, kind: str, dev: str):
+    def __init__(self, kind: str, dev: str, grouped: bool = True):
         import paper_2410_09687_b200 as moin
-        self.moin, self.kind, self.dev = moin, kind, dev
+        self.moin, self.kind, self.dev, self.grouped = moin, kind, dev, grouped
         if kind == "decode":
             self.E, self.r, self.T, self.R, self.K, self.seed = 500, 64, 256, 256, 500, 1
             self.mode = moin.PLAN_SEGMENTS
@@ -147,6 +148,12 @@ class LayerWorkload:
         self.plan = moin.Plan(self.T, self.E, dev, self.mode)
         ws = max(moin.lib().moin_lora_linear_workspace_bytes(self.T, d_in, d_out, self.r) for _, d_in, d_out in self.projs)
         self.ws = torch.empty(ws, dtype=torch.uint8, device=dev)
+        # projections that are independent inside a decoder block are issued as one grouped call
+        self.groups = GROUPS if grouped else [[p] for p in range(len(self.projs))]
+        self.jobgroups = [[moin.JobGroup([(self.x[p][i], self.W[p], self.pools[p], self.y[p]) for p in g])
+                           for g in self.groups] for i in range(ROTATE)]
+        self.ws = torch.empty(max(max(jg.workspace_bytes for jg in row) for row in self.jobgroups), dtype=torch.uint8,
+                              device=dev)
         # host-side staging for the end-to-end arm
         self.n_host = ROTATE if kind == "decode" else 1
         self.h_q = [q.cpu().pin_memory() for q in self.queries[:self.n_host]]
@@ -154,10 +161,12 @@ class LayerWorkload:
         self.h_y = [torch.empty_like(y, device="cpu").pin_memory() for y in self.y]
         self.d_q = torch.empty_like(self.queries[0])
         self.d_x = [torch.empty_like(xs[0]) for xs in self.x]
+        self.e2e_groups = [moin.JobGroup([(self.d_x[p], self.W[p], self.pools[p], self.y[p]) for p in g])
+                           for g in self.groups]
         self.h2d = self.d_q.numel() * 2 + sum(x.numel() * 2 for x in self.d_x)
         self.d2h = sum(y.numel() * 2 for y in self.y)
 
-    def _core(self, i: int, q, xs):
+    def _core(self, i: int, q, xs, jobgroups=None):
         moin = self.moin
         moin.route(self.routers[i], q, out_expert=self.req_expert)
         if self.kind == "decode":
@@ -167,12 +176,12 @@ class LayerWorkload:
             self.token_expert.view(self.R, L).copy_(self.req_expert.unsqueeze(1).expand(self.R, L))
             te = self.token_expert
         moin.plan_build(te, self.E, self.mode, plan=self.plan)
-        for p in range(len(self.projs)):
-            moin.lora_linear(self.plan, xs[p], self.W[p], self.pools[p], self.scale, y=self.y[p], workspace=self.ws)
+        for jg in jobgroups:
+            moin.lora_linear_group(self.plan, jg, self.scale, workspace=self.ws)
 
     def step(self, i: int):
         i %= ROTATE
-        self._core(i, self.queries[i], [xs[i] for xs in self.x])
+        self._core(i, self.queries[i], [xs[i] for xs in self.x], self.jobgroups[i])
 
     def step_e2e(self, i: int):
         i %= ROTATE
@@ -180,7 +189,7 @@ class LayerWorkload:
         self.d_q.copy_(self.h_q[j], non_blocking=True)
         for p in range(len(self.projs)):
             self.d_x[p].copy_(self.h_x[p][j], non_blocking=True)
-        self._core(i, self.d_q, self.d_x)
+        self._core(i, self.d_q, self.d_x, self.e2e_groups)
         for p in range(len(self.projs)):
             self.h_y[p].copy_(self.y[p], non_blocking=True)
 
@@ -209,7 +218,8 @@ class LayerWorkload:
         name = ("decode: 7 TinyLlama projections, 500 experts rank 64, 256 single tokens, router 256x500x768"
                 if self.kind == "decode" else
                 "prefill: 7 TinyLlama projections, 5000 experts rank 16, 32x512 tokens Zipf(1.1), router 32x5000x768")
-        return {"workload": name, "tokens_per_step": self.T, "experts": self.E, "rank": self.r, "lora_scale": self.scale,
+        return {"workload": name, "calls": ("grouped {q,k,v} {o} {gate,up} {down}" if self.grouped else "one call per projection"),
+                "tokens_per_step": self.T, "experts": self.E, "rank": self.r, "lora_scale": self.scale,
                 "l2": f"inputs rotate over {ROTATE} batches; per-step working set exceeds L2"}
 
     def oracle_sample(self, n_tokens: int) -> float:
@@ -514,6 +524,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-router-extra", action="store_true")
     ap.add_argument("--forward-layers", type=int, default=22)
+    ap.add_argument("--no-group", action="store_true", help="one moin_lora_linear call per projection")
     ap.add_argument("--stream-impl", type=int, default=0, help="short-segment LoRA kernels: 0 auto, 1 register-fed, 2 TMA-staged")
     args = ap.parse_args()
     defaults = {"decode": (3000, 20), "prefill": (100, 5), "router": (50, 5), "forward": (5, 3)}
@@ -539,7 +550,7 @@ def main():
     peaks = load_peaks()
     kind = args.workload
     if kind in ("decode", "prefill"):
-        wl = LayerWorkload(kind, dev)
+        wl = LayerWorkload(kind, dev, grouped=not args.no_group)
     elif kind == "router":
         wl = RouterWorkload(dev)
     else:
@@ -582,7 +593,7 @@ def main():
         name_to_key = {"lora_expand_stream": "expand", "lora_shrink_stream": "shrink", "gemm_warp": "gemm", "gemm_tc": "gemm"}
         if top in name_to_key:
             a = agg[top]
-            bytes_per_launch = alg["per_kernel_bytes"][name_to_key[top]] / len(wl.projs)
+            bytes_per_launch = alg["per_kernel_bytes"][name_to_key[top]] * prof_steps / a["launches"]
             sec = a["ms"] * 1e-3 / a["launches"]
             ach = bytes_per_launch / sec / 1e9
             roof = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -591,7 +602,7 @@ def main():
                     "traffic": traffic_for(top, kind)}
         elif top in ("lora_fused_tc", "lora_shrink_tc"):
             a = agg[top]
-            fl = alg["step_flops"] / len(wl.projs)
+            fl = alg["step_flops"] * prof_steps / a["launches"]
             sec = a["ms"] * 1e-3 / a["launches"]
             ach = fl / sec / 1e12
             roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],

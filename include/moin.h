@@ -225,6 +225,24 @@ moin_status moin_lora_linear(const moin_plan* plan, const void* x, const void* W
                              float scale, int32_t base_T, int32_t base_d_in, int32_t base_d_out, void* y,
                              void* workspace, size_t workspace_bytes, moin_stream stream);
 
+/* Grouped form: up to MOIN_MAX_GROUP projections that share the batch plan and do not depend on one
+ * another - in a decoder block {q, k, v} and {gate, up} (paper Sec. 3.2: the adapter sits on every linear
+ * layer, so independent layers of a block can be served together).  The result of every job is exactly
+ * that of moin_lora_linear on it; the group exists because in the short-segment (decode) regime the
+ * kernels are bound by adapter streaming plus a fixed per-launch cost, and one merged shrink and one
+ * merged expand launch pay that cost once per group.  Every job needs a pool; the jobs' x, W, y follow
+ * the rules of moin_lora_linear.  Workspace: moin_lora_linear_group_workspace_bytes. */
+enum { MOIN_MAX_GROUP = 4 };
+typedef struct {
+  const void* x;          /* [T, pool->d_in] bf16 */
+  const void* W;          /* [pool->d_out, pool->d_in] bf16 */
+  const moin_pool* pool;  /* adapters of this projection */
+  void* y;                /* [T, pool->d_out] bf16 */
+} moin_lora_job;
+size_t moin_lora_linear_group_workspace_bytes(int32_t T, const moin_lora_job* jobs, int32_t n_jobs);
+moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* jobs, int32_t n_jobs, float scale,
+                                   void* workspace, size_t workspace_bytes, moin_stream stream);
+
 /* ---------------------------------------------------------------------------------------
  * Decoder forward.  Paper Sec. 4: the base model is TinyLlama-1.1B (Llama-2 architecture);
  * Sec. 3.2: an adapter on each linear layer; Sec. 3.3: the request's expert for the whole

@@ -22,7 +22,7 @@ EXPORTED_SYMBOLS = (
     "moin_set_option", "moin_router_prepare", "moin_route_workspace_bytes", "moin_route", "moin_plan_bytes",
     "moin_plan_build", "moin_plan_read", "moin_lora_linear_workspace_bytes", "moin_lora_linear",
     "moin_decoder_workspace_bytes", "moin_decoder_forward", "moin_profile_enable", "moin_profile_read",
-    "moin_kernel_name", "moin_route_static",
+    "moin_kernel_name", "moin_route_static", "moin_lora_linear_group", "moin_lora_linear_group_workspace_bytes",
 )
 
 
@@ -39,6 +39,10 @@ class _Pool(ctypes.Structure):
     _fields_ = [("A", ctypes.c_void_p), ("B", ctypes.c_void_p), ("slot_of_expert", ctypes.c_void_p),
                 ("E", ctypes.c_int32), ("n_slots", ctypes.c_int32), ("r", ctypes.c_int32), ("d_in", ctypes.c_int32),
                 ("d_out", ctypes.c_int32)]
+
+
+class _Job(ctypes.Structure):
+    _fields_ = [("x", ctypes.c_void_p), ("W", ctypes.c_void_p), ("pool", ctypes.POINTER(_Pool)), ("y", ctypes.c_void_p)]
 
 
 class _Plan(ctypes.Structure):
@@ -102,6 +106,9 @@ def lib() -> ctypes.CDLL:
         L.moin_lora_linear_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.moin_lora_linear.argtypes = [ctypes.POINTER(_Plan), vp, vp, ctypes.POINTER(_Pool), f32, i32, i32, i32, vp,
                                        vp, sz, vp]
+        L.moin_lora_linear_group_workspace_bytes.restype = sz
+        L.moin_lora_linear_group_workspace_bytes.argtypes = [i32, ctypes.POINTER(_Job), i32]
+        L.moin_lora_linear_group.argtypes = [ctypes.POINTER(_Plan), ctypes.POINTER(_Job), i32, f32, vp, sz, vp]
         L.moin_decoder_workspace_bytes.restype = sz
         L.moin_decoder_workspace_bytes.argtypes = [ctypes.POINTER(_Model), i32, i32]
         L.moin_decoder_forward.argtypes = [ctypes.POINTER(_Model), vp, vp, vp, i32, i32, i32, vp, i32,
@@ -308,6 +315,33 @@ def lora_linear(plan: Optional[Plan], x: torch.Tensor, W: torch.Tensor, pool: Op
                                   ctypes.byref(pool.c) if use else None, float(scale), T, d_in, d_out, _ptr(y),
                                   _ptr(ws), ws.numel(), _stream(stream)), "moin_lora_linear")
     return y
+
+
+class JobGroup:
+    """moin_lora_job array for moin_lora_linear_group: up to 4 independent projections sharing one plan.
+
+    ``jobs``: sequence of (x, W, pool, y) with y preallocated (bf16 [T, d_out])."""
+
+    def __init__(self, jobs: Sequence[tuple]):
+        assert 1 <= len(jobs) <= 4
+        self._keep = list(jobs)
+        self.n = len(jobs)
+        self.c = (_Job * self.n)()
+        for i, (x, W, pool, y) in enumerate(jobs):
+            assert x.dtype == torch.bfloat16 and W.dtype == torch.bfloat16 and y.dtype == torch.bfloat16
+            assert x.shape[1] == pool.d_in and W.shape == (pool.d_out, pool.d_in) and y.shape == (x.shape[0], pool.d_out)
+            self.c[i] = _Job(_ptr(x), _ptr(W), ctypes.pointer(pool.c), _ptr(y))
+        self.T = jobs[0][0].shape[0]
+        self.device = jobs[0][0].device
+        self.workspace_bytes = lib().moin_lora_linear_group_workspace_bytes(self.T, self.c, self.n)
+
+
+def lora_linear_group(plan: Plan, group: JobGroup, scale: float, workspace: Optional[torch.Tensor] = None,
+                      stream=None) -> None:
+    """moin_lora_linear_group: every job's y = x W^T + scale (x A_e^T) B_e^T, merged launches."""
+    ws = workspace if workspace is not None else _workspace(group.device, group.workspace_bytes)
+    _check(lib().moin_lora_linear_group(ctypes.byref(plan.c), group.c, group.n, float(scale), _ptr(ws), ws.numel(),
+                                        _stream(stream)), "moin_lora_linear_group")
 
 
 PROJ_ORDER = ("q", "k", "v", "o", "gate", "up", "down")

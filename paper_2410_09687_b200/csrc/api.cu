@@ -30,10 +30,12 @@ moin_status host_state(HostState** out) {
     e = cudaGetSymbolAddress(&p, g_device_status);
     if (e != cudaSuccess) return record_cuda(e);
     g_state.status = reinterpret_cast<DeviceStatus*>(p);
-    if (g_state.side == nullptr) {
-      e = cudaStreamCreateWithFlags(&g_state.side, cudaStreamNonBlocking);
-      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_state.ev_fork, cudaEventDisableTiming);
-      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_state.ev_join, cudaEventDisableTiming);
+    if (g_state.ev_fork == nullptr) {
+      e = cudaEventCreateWithFlags(&g_state.ev_fork, cudaEventDisableTiming);
+      for (int j = 0; j < kMaxStreamJobs && e == cudaSuccess; ++j) {
+        e = cudaStreamCreateWithFlags(&g_state.side[j], cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g_state.ev_join[j], cudaEventDisableTiming);
+      }
       if (e != cudaSuccess) return record_cuda(e);
     }
     g_state.n_sms = prop.multiProcessorCount;
@@ -352,93 +354,182 @@ size_t moin_lora_linear_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, 
   return (seg > tiles ? seg : tiles) + 256;
 }
 
-moin_status moin_lora_linear(const moin_plan* plan, const void* x, const void* W, const moin_pool* pool,
-                             float scale, int32_t base_T, int32_t base_d_in, int32_t base_d_out, void* y,
-                             void* workspace, size_t workspace_bytes, moin_stream stream) {
-  const bool lora = (plan != nullptr && pool != nullptr);
-  const int T = lora ? plan->T : base_T;
-  const int d_in = lora ? pool->d_in : base_d_in;
-  const int d_out = lora ? pool->d_out : base_d_out;
-  if (T < 0) return MOIN_ERR_INVALID_ARG;
-  if (T == 0) return MOIN_OK;
+// Checks one projection job; fills T / d_in / d_out / r.  `lora` = the job carries an adapter pool.
+static moin_status check_job(const moin_plan* plan, const void* x, const void* W, const moin_pool* pool, const void* y,
+                             bool lora, int base_T, int base_d_in, int base_d_out, int* T, int* d_in, int* d_out,
+                             int* r) {
+  *T = lora ? plan->T : base_T;
+  *d_in = lora ? pool->d_in : base_d_in;
+  *d_out = lora ? pool->d_out : base_d_out;
+  *r = 0;
+  if (*T < 0) return MOIN_ERR_INVALID_ARG;
+  if (*T == 0) return MOIN_OK;
   if (!x || !W || !y || x == y) return MOIN_ERR_INVALID_ARG;
-  if (d_in < 64 || (d_in % 64) != 0 || d_out < 8 || (d_out % 8) != 0) return MOIN_ERR_BAD_SHAPE;
+  if (*d_in < 64 || (*d_in % 64) != 0 || *d_out < 8 || (*d_out % 8) != 0) return MOIN_ERR_BAD_SHAPE;
   if (!aligned16(x) || !aligned16(W) || !aligned16(y)) return MOIN_ERR_MISALIGNED;
-  int r = 0;
   if (lora) {
-    r = pool->r;
-    if (r < 8 || r > 64 || (r % 8) != 0) return MOIN_ERR_UNSUPPORTED_RANK;
+    *r = pool->r;
+    if (*r < 8 || *r > 64 || (*r % 8) != 0) return MOIN_ERR_UNSUPPORTED_RANK;
     if (!pool->A || !pool->B || !pool->slot_of_expert || !plan->buffer) return MOIN_ERR_INVALID_ARG;
     if (pool->E != plan->E) return MOIN_ERR_INVALID_ARG;
     if (!aligned16(pool->A) || !aligned16(pool->B)) return MOIN_ERR_MISALIGNED;
     if (plan->mode != MOIN_PLAN_SEGMENTS && plan->mode != MOIN_PLAN_TILES) return MOIN_ERR_INVALID_ARG;
   }
+  return MOIN_OK;
+}
+
+static moin_status pick_gemm(const HostState* hs, int T, int d_in, int d_out, bool* use_tc) {
+  const bool tc_ok = tc_gemm_supported(T, d_in, d_out);
+  *use_tc = tc_ok && T >= 64 && d_out >= 64;
+  if (hs->gemm_impl == 1) *use_tc = false;
+  if (hs->gemm_impl == 2) {
+    if (!tc_ok) return MOIN_ERR_BAD_SHAPE;
+    *use_tc = true;
+  }
+  return MOIN_OK;
+}
+
+size_t moin_lora_linear_group_workspace_bytes(int32_t T, const moin_lora_job* jobs, int32_t n_jobs) {
+  size_t total = 0;   // the per-projection sizes are multiples of 256 and carry their own slack
+  for (int j = 0; jobs && j < n_jobs; ++j)
+    if (jobs[j].pool)
+      total += align_up(moin_lora_linear_workspace_bytes(T, jobs[j].pool->d_in, jobs[j].pool->d_out, jobs[j].pool->r), 256);
+  return total;
+}
+
+moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* jobs, int32_t n_jobs, float scale,
+                                   void* workspace, size_t workspace_bytes, moin_stream stream) {
+  if (!plan || !jobs || n_jobs < 1 || n_jobs > MOIN_MAX_GROUP) return MOIN_ERR_INVALID_ARG;
+  int T = 0, d_in[kMaxStreamJobs], d_out[kMaxStreamJobs], r[kMaxStreamJobs];
+  for (int j = 0; j < n_jobs; ++j) {
+    if (!jobs[j].pool) return MOIN_ERR_INVALID_ARG;
+    moin_status st = check_job(plan, jobs[j].x, jobs[j].W, jobs[j].pool, jobs[j].y, true, 0, 0, 0, &T, &d_in[j],
+                               &d_out[j], &r[j]);
+    if (st) return st;
+  }
+  if (T == 0) return MOIN_OK;
   HostState* hs;
   moin_status st = host_state(&hs);
   if (st) return st;
-  cudaStream_t s = (cudaStream_t)stream;
-  const __nv_bfloat16* xb = (const __nv_bfloat16*)x;
-  const __nv_bfloat16* Wb = (const __nv_bfloat16*)W;
-  __nv_bfloat16* yb = (__nv_bfloat16*)y;
-
-  const bool tc_ok = tc_gemm_supported(T, d_in, d_out);
-  bool use_tc = tc_ok && T >= 64 && d_out >= 64;
-  if (hs->gemm_impl == 1) use_tc = false;
-  if (hs->gemm_impl == 2) {
-    if (!tc_ok) return MOIN_ERR_BAD_SHAPE;
-    use_tc = true;
-  }
-
-  if (!lora) {
-    ProfScope prof(use_tc ? MOIN_K_GEMM_TC : MOIN_K_GEMM_WARP, 1, s);
-    if (use_tc) return launch_tc_gemm(hs, xb, Wb, yb, nullptr, T, d_in, d_out, s);
-    return record_cuda(launch_gemm_warp(xb, Wb, yb, nullptr, T, d_in, d_out, s));
-  }
-  if (!workspace || !aligned16(workspace) || workspace_bytes < moin_lora_linear_workspace_bytes(T, d_in, d_out, r))
+  if (!workspace || !aligned16(workspace) || workspace_bytes < moin_lora_linear_group_workspace_bytes(T, jobs, n_jobs))
     return MOIN_ERR_WORKSPACE;
+  cudaStream_t s = (cudaStream_t)stream;
   PlanView pv = plan_view(plan->buffer, plan->T, plan->E);
   char* ws = reinterpret_cast<char*>(workspace);
+  char* ws_job[kMaxStreamJobs];
+  bool use_tc[kMaxStreamJobs];
+  for (int j = 0; j < n_jobs; ++j) {
+    ws_job[j] = ws;
+    ws += align_up(moin_lora_linear_workspace_bytes(T, d_in[j], d_out[j], r[j]), 256);
+    if ((st = pick_gemm(hs, T, d_in[j], d_out[j], &use_tc[j]))) return st;
+  }
 
-  if (plan->mode == MOIN_PLAN_TILES && use_tc && tc_fused_supported(r)) {
-    __nv_bfloat16* hb = reinterpret_cast<__nv_bfloat16*>(ws);  // [T, r] bf16, s * (x A^T)
-    return launch_tc_lora_tiles(hs, pv, pool, xb, Wb, yb, hb, scale, s);
+  if (plan->mode == MOIN_PLAN_TILES) {
+    // Long runs: every projection is one grouped-shrink + one fused GEMM launch on the tensor cores.
+    bool all_tc = true;
+    for (int j = 0; j < n_jobs; ++j) all_tc = all_tc && use_tc[j] && tc_fused_supported(r[j]);
+    if (all_tc) {
+      for (int j = 0; j < n_jobs; ++j) {
+        st = launch_tc_lora_tiles(hs, pv, jobs[j].pool, (const __nv_bfloat16*)jobs[j].x, (const __nv_bfloat16*)jobs[j].W,
+                                  (__nv_bfloat16*)jobs[j].y, reinterpret_cast<__nv_bfloat16*>(ws_job[j]), scale, s);
+        if (st) return st;
+      }
+      return MOIN_OK;
+    }
   }
-  // Short segments: the base GEMM (y and fp32 y0) and the shrink are independent, so the GEMM runs on
-  // the library's side stream between a fork and a join event; the expand then adds y0 + s h B^T.
-  const bool tma_stream = hs->stream_impl != 1;                 // MOIN_OPT_STREAM_IMPL
-  const bool tma_shrink = tma_stream && lora_shrink_tma_supported(d_in);
-  const int parts = tma_shrink ? lora_stream_parts(d_in) : 1;
-  float* h = reinterpret_cast<float*>(ws);                      // [parts][T][r] partial shrink results
-  float* y0 = reinterpret_cast<float*>(ws + align_up((size_t)lora_stream_parts(d_in) * (size_t)T * (size_t)r * sizeof(float), 256));
+  // Short segments.  Per projection: y0 = x W^T (fp32 + bf16 copy), h = x A_e^T, y = bf16(y0 + s h B_e^T).
+  // The base GEMMs do not depend on the shrink, so each runs on one of the library's side streams between
+  // a fork and a join event, concurrently with the shrink; the shrink and the expand each cover all the
+  // projections of the group in ONE launch, so their launch and ramp-up costs are paid once per group.
+  float* h[kMaxStreamJobs];
+  float* y0[kMaxStreamJobs];
+  int parts[kMaxStreamJobs];
+  const bool tma_stream = hs->stream_impl == 2 && n_jobs == 1;   // MOIN_OPT_STREAM_IMPL: TMA-staged kernels (one job)
+  for (int j = 0; j < n_jobs; ++j) {
+    parts[j] = (tma_stream && lora_shrink_tma_supported(d_in[j])) ? lora_stream_parts(d_in[j]) : 1;
+    h[j] = reinterpret_cast<float*>(ws_job[j]);   // [parts][T][r] (partial) shrink results
+    y0[j] = reinterpret_cast<float*>(ws_job[j] + align_up((size_t)lora_stream_parts(d_in[j]) * (size_t)T * (size_t)r[j] * sizeof(float), 256));
+  }
   cudaError_t ce = cudaEventRecord(hs->ev_fork, s);
-  if (ce == cudaSuccess) ce = cudaStreamWaitEvent(hs->side, hs->ev_fork, 0);
   if (ce != cudaSuccess) return record_cuda(ce);
-  {
-    ProfScope prof(use_tc ? MOIN_K_GEMM_TC : MOIN_K_GEMM_WARP, 1, hs->side);
-    if (use_tc)
-      st = launch_tc_gemm(hs, xb, Wb, yb, y0, T, d_in, d_out, hs->side);
+  moin_status st_gemm = MOIN_OK;
+  for (int j = 0; j < n_jobs; ++j) {
+    ce = cudaStreamWaitEvent(hs->side[j], hs->ev_fork, 0);
+    if (ce != cudaSuccess) return record_cuda(ce);
+    ProfScope prof(use_tc[j] ? MOIN_K_GEMM_TC : MOIN_K_GEMM_WARP, 1, hs->side[j]);
+    moin_status sj;
+    if (use_tc[j])
+      sj = launch_tc_gemm(hs, (const __nv_bfloat16*)jobs[j].x, (const __nv_bfloat16*)jobs[j].W, (__nv_bfloat16*)jobs[j].y,
+                          y0[j], T, d_in[j], d_out[j], hs->side[j]);
     else
-      st = record_cuda(launch_gemm_warp(xb, Wb, yb, y0, T, d_in, d_out, hs->side));
+      sj = record_cuda(launch_gemm_warp((const __nv_bfloat16*)jobs[j].x, (const __nv_bfloat16*)jobs[j].W,
+                                        (__nv_bfloat16*)jobs[j].y, y0[j], T, d_in[j], d_out[j], hs->side[j]));
+    if (sj && !st_gemm) st_gemm = sj;
   }
-  moin_status st2;
+  moin_status st_shrink;
   {
     ProfScope prof(MOIN_K_SHRINK_STREAM, 1, s);
-    if (tma_shrink)
-      st2 = launch_lora_shrink_tma(hs, pv, pool, xb, h, s);
-    else
-      st2 = record_cuda(launch_lora_shrink_stream(pv, pool->slot_of_expert, xb, (const __nv_bfloat16*)pool->A, h, r,
-                                                  d_in, hs->n_sms, s));
+    if (tma_stream && parts[0] >= 1 && lora_shrink_tma_supported(d_in[0])) {
+      st_shrink = launch_lora_shrink_tma(hs, pv, jobs[0].pool, (const __nv_bfloat16*)jobs[0].x, h[0], s);
+    } else {
+      ShrinkJobs sj = {};
+      sj.n = n_jobs;
+      for (int j = 0; j < n_jobs; ++j) {
+        sj.x[j] = (const __nv_bfloat16*)jobs[j].x;
+        sj.A[j] = (const __nv_bfloat16*)jobs[j].pool->A;
+        sj.h[j] = h[j];
+        sj.slot_of_expert[j] = jobs[j].pool->slot_of_expert;
+        sj.r[j] = r[j];
+        sj.d_in[j] = d_in[j];
+      }
+      st_shrink = record_cuda(launch_lora_shrink_stream(pv, sj, hs->n_sms, s));
+    }
   }
-  // always join, even after a failed launch, so the side stream never outlives the call's ordering
-  ce = cudaEventRecord(hs->ev_join, hs->side);
-  if (ce == cudaSuccess) ce = cudaStreamWaitEvent(s, hs->ev_join, 0);
-  if (st) return st;
-  if (st2) return st2;
-  if (ce != cudaSuccess) return record_cuda(ce);
+  // always join, even after a failed launch, so the side streams never outlive the call's ordering
+  for (int j = 0; j < n_jobs; ++j) {
+    ce = cudaEventRecord(hs->ev_join[j], hs->side[j]);
+    if (ce == cudaSuccess) ce = cudaStreamWaitEvent(s, hs->ev_join[j], 0);
+    if (ce != cudaSuccess) return record_cuda(ce);
+  }
+  if (st_gemm) return st_gemm;
+  if (st_shrink) return st_shrink;
   ProfScope prof(MOIN_K_EXPAND_STREAM, 1, s);
-  if (tma_stream) return launch_lora_expand_tma(hs, pv, pool, h, parts, y0, yb, scale, s);
-  return record_cuda(launch_lora_expand_stream(pv, pool->slot_of_expert, h, (const __nv_bfloat16*)pool->B, y0, yb,
-                                               scale, r, d_out, hs->n_sms, s));
+  if (tma_stream) return launch_lora_expand_tma(hs, pv, jobs[0].pool, h[0], parts[0], y0[0], (__nv_bfloat16*)jobs[0].y, scale, s);
+  ExpandJobs ej = {};
+  ej.n = n_jobs;
+  for (int j = 0; j < n_jobs; ++j) {
+    ej.h[j] = h[j];
+    ej.B[j] = (const __nv_bfloat16*)jobs[j].pool->B;
+    ej.y0[j] = y0[j];
+    ej.y[j] = (__nv_bfloat16*)jobs[j].y;
+    ej.slot_of_expert[j] = jobs[j].pool->slot_of_expert;
+    ej.r[j] = r[j];
+    ej.d_out[j] = d_out[j];
+  }
+  return record_cuda(launch_lora_expand_stream(pv, ej, scale, hs->n_sms, s));
+}
+
+moin_status moin_lora_linear(const moin_plan* plan, const void* x, const void* W, const moin_pool* pool,
+                             float scale, int32_t base_T, int32_t base_d_in, int32_t base_d_out, void* y,
+                             void* workspace, size_t workspace_bytes, moin_stream stream) {
+  const bool lora = (plan != nullptr && pool != nullptr);
+  if (lora) {   // one-job group
+    moin_lora_job job = {x, W, pool, y};
+    if (plan->T > 0 && workspace_bytes < moin_lora_linear_workspace_bytes(plan->T, pool->d_in, pool->d_out, pool->r))
+      return MOIN_ERR_WORKSPACE;
+    return moin_lora_linear_group(plan, &job, 1, scale, workspace, workspace_bytes, stream);
+  }
+  int T, d_in, d_out, r;
+  moin_status st = check_job(plan, x, W, pool, y, false, base_T, base_d_in, base_d_out, &T, &d_in, &d_out, &r);
+  if (st || T == 0) return st;
+  HostState* hs;
+  if ((st = host_state(&hs))) return st;
+  bool use_tc;
+  if ((st = pick_gemm(hs, T, d_in, d_out, &use_tc))) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  ProfScope prof(use_tc ? MOIN_K_GEMM_TC : MOIN_K_GEMM_WARP, 1, s);
+  if (use_tc) return launch_tc_gemm(hs, (const __nv_bfloat16*)x, (const __nv_bfloat16*)W, (__nv_bfloat16*)y, nullptr, T, d_in, d_out, s);
+  return record_cuda(launch_gemm_warp((const __nv_bfloat16*)x, (const __nv_bfloat16*)W, (__nv_bfloat16*)y, nullptr, T, d_in, d_out, s));
 }
 
 }  // extern "C"

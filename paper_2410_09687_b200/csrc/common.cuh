@@ -109,12 +109,28 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // Launchers implemented in the .cu files (host side).
 cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, DeviceStatus* status, cudaStream_t stream);
-cudaError_t launch_lora_shrink_stream(const PlanView& pv, const int* slot_of_expert, const __nv_bfloat16* x,
-                                      const __nv_bfloat16* A, float* h, int r, int d_in, int n_sms,
+// Register-fed short-segment kernels: one launch covers up to kMaxStreamJobs projections sharing a plan.
+constexpr int kMaxStreamJobs = 4;
+struct ShrinkJobs {
+  const __nv_bfloat16* x[kMaxStreamJobs];
+  const __nv_bfloat16* A[kMaxStreamJobs];
+  float* h[kMaxStreamJobs];
+  const int* slot_of_expert[kMaxStreamJobs];
+  int r[kMaxStreamJobs], d_in[kMaxStreamJobs], per_seg[kMaxStreamJobs];
+  int n;
+};
+struct ExpandJobs {
+  const float* h[kMaxStreamJobs];
+  const __nv_bfloat16* B[kMaxStreamJobs];
+  const float* y0[kMaxStreamJobs];
+  __nv_bfloat16* y[kMaxStreamJobs];
+  const int* slot_of_expert[kMaxStreamJobs];
+  int r[kMaxStreamJobs], d_out[kMaxStreamJobs], rows_per_item[kMaxStreamJobs], per_seg[kMaxStreamJobs];
+  int n;
+};
+cudaError_t launch_lora_shrink_stream(const PlanView& pv, ShrinkJobs jobs, int n_sms, cudaStream_t stream);
+cudaError_t launch_lora_expand_stream(const PlanView& pv, ExpandJobs jobs, float scale, int n_sms,
                                       cudaStream_t stream);
-cudaError_t launch_lora_expand_stream(const PlanView& pv, const int* slot_of_expert, const float* h,
-                                      const __nv_bfloat16* B, const float* y0, __nv_bfloat16* y, float scale, int r,
-                                      int d_out, int n_sms, cudaStream_t stream);
 cudaError_t launch_gemm_warp(const __nv_bfloat16* x, const __nv_bfloat16* W, __nv_bfloat16* y, float* y0, int T,
                              int d_in, int d_out, cudaStream_t stream);
 cudaError_t launch_inv_norm(const __nv_bfloat16* c, int K, int D, float* inv_norm, cudaStream_t stream);
@@ -132,8 +148,8 @@ struct HostState {
   int gemm_impl = 0;               // MOIN_OPT_GEMM_IMPL
   int stream_impl = 0;             // MOIN_OPT_STREAM_IMPL
   // fork/join inside one call: independent kernels of a call run on `side` between two events
-  cudaStream_t side = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  cudaStream_t side[kMaxStreamJobs] = {nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t ev_fork = nullptr, ev_join[kMaxStreamJobs] = {nullptr, nullptr, nullptr, nullptr};
 };
 moin_status host_state(HostState** out);      // lazily initialised for the current device
 moin_status record_cuda(cudaError_t e);       // MOIN_OK or MOIN_ERR_CUDA (remembers e)

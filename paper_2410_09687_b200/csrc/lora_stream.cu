@@ -19,41 +19,79 @@ constexpr int kShrinkUnroll = 8;         // 32-wide k steps in flight per warp
 constexpr int kExpandThreads = 128;      // 4 warps
 constexpr int kExpandTilesPerBatch = 2;  // 16-row tiles whose loads are in flight together, per warp
 
-struct SegMeta { int slot, s0, n; };
-__device__ __forceinline__ SegMeta load_seg(const int* __restrict__ seg_expert, const int* __restrict__ seg_start,
-                                            const int* __restrict__ slot_of_expert, int seg, bool valid) {
-  SegMeta m = {-1, 0, 0};
-  if (valid) {
-    m.slot = slot_of_expert[seg_expert[seg]];
-    m.s0 = seg_start[seg];
-    m.n = seg_start[seg + 1] - m.s0;
+// Work items of a launch span up to kMaxStreamJobs projections that share one batch plan: item index ->
+// (job, segment, sub-block), jobs laid out one after the other, `per_seg[j]` items per segment in job j.
+// Kernel parameters are only ever indexed with compile-time indices (a run-time index would force a
+// local-memory copy of the parameter block): pick(arr, j) selects arr[j] with a compare chain.
+template <class V>
+__device__ __forceinline__ V pick(const V (&arr)[kMaxStreamJobs], int j) {
+  V v = arr[0];
+#pragma unroll
+  for (int i = 1; i < kMaxStreamJobs; ++i)
+    if (j == i) v = arr[i];
+  return v;
+}
+
+struct ItemRef { int job, seg, sub; };
+template <class Jobs>
+__device__ __forceinline__ ItemRef decode_item(int item, int nseg, const Jobs& jobs) {
+  ItemRef it = {0, 0, 0};
+  int rem = item;
+#pragma unroll
+  for (int j = 0; j + 1 < kMaxStreamJobs; ++j) {
+    if (it.job == j && j + 1 < jobs.n && rem >= nseg * jobs.per_seg[j]) {
+      rem -= nseg * jobs.per_seg[j];
+      it.job = j + 1;
+    }
+  }
+  const int ps = pick(jobs.per_seg, it.job);
+  it.seg = rem / ps;
+  it.sub = rem - it.seg * ps;
+  return it;
+}
+
+struct SegMeta { int slot, s0, n, job, sub; };
+template <class Jobs>
+__device__ __forceinline__ SegMeta load_seg(const int4* __restrict__ seg_tab, const Jobs& jobs, int item, int items,
+                                            int nseg) {
+  SegMeta m = {-1, 0, 0, 0, 0};
+  if (item < items) {
+    const ItemRef it = decode_item(item, nseg, jobs);
+    const int4 e = __ldg(seg_tab + it.seg);   // (expert, start, length, -)
+    m.slot = __ldg(pick(jobs.slot_of_expert, it.job) + e.x);
+    m.s0 = e.y;
+    m.n = e.z;
+    m.job = it.job;
+    m.sub = it.sub;
   }
   return m;
 }
 
 // h[pos][rho] = sum_i A[slot][rho][i] * x[perm[pos]][i]      (fp32, pos = position in sorted order)
-// Work item = (segment, group of 16 adapter rows); the CTA's 8 warps interleave over k.
+// Work item = (job, segment, group of 16 adapter rows); the CTA's 8 warps interleave over k.
 __global__ void __launch_bounds__(kShrinkThreads, 2)
 lora_shrink_stream_kernel(const int* __restrict__ header, const int* __restrict__ perm,
-                          const int* __restrict__ seg_expert, const int* __restrict__ seg_start,
-                          const int* __restrict__ slot_of_expert, const __nv_bfloat16* __restrict__ x,
-                          const __nv_bfloat16* __restrict__ A, float* __restrict__ h, int r, int d_in) {
+                          const int4* __restrict__ seg_tab, const ShrinkJobs jobs) {
   __shared__ float red[kShrinkWarps][32][4];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int nseg = header[PH_NSEG];
-  const int MG = (r + 15) >> 4;
-  const int steps = d_in >> 5;  // 32 k per step
-  const int items = nseg * MG;
+  int items = 0;
+#pragma unroll
+  for (int j = 0; j < kMaxStreamJobs; ++j)
+    if (j < jobs.n) items += nseg * jobs.per_seg[j];
   int item = blockIdx.x;
-  SegMeta nxt = load_seg(seg_expert, seg_start, slot_of_expert, item / MG, item < items);
+  SegMeta nxt = load_seg(seg_tab, jobs, item, items, nseg);
   for (; item < items; item += gridDim.x) {
     const SegMeta cur = nxt;
-    const int mg = item % MG;
-    const int ni = item + gridDim.x;
-    nxt = load_seg(seg_expert, seg_start, slot_of_expert, ni / MG, ni < items);  // one item of lookahead
+    nxt = load_seg(seg_tab, jobs, item + gridDim.x, items, nseg);  // lookahead
     if (cur.slot < 0) continue;  // uniform per CTA
-    const int rho0 = mg * 16 + g, rho1 = rho0 + 8;
+    const int r = pick(jobs.r, cur.job), d_in = pick(jobs.d_in, cur.job);
+    const __nv_bfloat16* __restrict__ x = pick(jobs.x, cur.job);
+    const __nv_bfloat16* __restrict__ A = pick(jobs.A, cur.job);
+    float* __restrict__ h = pick(jobs.h, cur.job);
+    const int steps = d_in >> 5;  // 32 k per step
+    const int rho0 = cur.sub * 16 + g, rho1 = rho0 + 8;
     const bool v0 = rho0 < r, v1 = rho1 < r;
     const __nv_bfloat16* a_row0 = A + ((size_t)cur.slot * r + (v0 ? rho0 : 0)) * (size_t)d_in + 8 * t;
     const __nv_bfloat16* a_row1 = A + ((size_t)cur.slot * r + (v1 ? rho1 : 0)) * (size_t)d_in + 8 * t;
@@ -116,31 +154,33 @@ lora_shrink_stream_kernel(const int* __restrict__ header, const int* __restrict_
 
 // y[perm[pos]][j] = bf16( y0[perm[pos]][j] + scale * sum_rho B[slot][j][rho] * h[pos][rho] )
 // h is split into bf16 hi + lo parts (two MMAs) so the low-rank term keeps ~fp32 accuracy.
-// Work item = (segment, block of rows_per_item output features); each warp walks its 16-row tiles
+// Work item = (job, segment, block of rows_per_item output features); each warp walks its 16-row tiles
 // kExpandTilesPerBatch at a time with the adapter rows and the base values y0 loaded together.
-template <int P>  // number of 32-wide rho groups: ceil(r / 32)
+template <int P>  // number of 32-wide rho groups: ceil(max r / 32)
 __global__ void __launch_bounds__(kExpandThreads, 4)
 lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict__ perm,
-                          const int* __restrict__ seg_expert, const int* __restrict__ seg_start,
-                          const int* __restrict__ slot_of_expert, const float* __restrict__ h,
-                          const __nv_bfloat16* __restrict__ B, const float* __restrict__ y0,
-                          __nv_bfloat16* __restrict__ y, float scale, int r, int d_out, int rows_per_item) {
+                          const int4* __restrict__ seg_tab, const ExpandJobs jobs, float scale) {
   constexpr int TB = kExpandTilesPerBatch;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int nseg = header[PH_NSEG];
-  const int JB = (d_out + rows_per_item - 1) / rows_per_item;
-  const int tiles_per_item = rows_per_item >> 4;
-  const int items = nseg * JB;
+  int items = 0;
+#pragma unroll
+  for (int j = 0; j < kMaxStreamJobs; ++j)
+    if (j < jobs.n) items += nseg * jobs.per_seg[j];
   int item = blockIdx.x;
-  SegMeta nxt = load_seg(seg_expert, seg_start, slot_of_expert, item / JB, item < items);
+  SegMeta nxt = load_seg(seg_tab, jobs, item, items, nseg);
   for (; item < items; item += gridDim.x) {
     const SegMeta cur = nxt;
-    const int jb = item % JB;
-    const int ni = item + gridDim.x;
-    nxt = load_seg(seg_expert, seg_start, slot_of_expert, ni / JB, ni < items);
+    nxt = load_seg(seg_tab, jobs, item + gridDim.x, items, nseg);
     if (cur.slot < 0) continue;
-    const __nv_bfloat16* Bs = B + (size_t)cur.slot * (size_t)d_out * (size_t)r;
+    const int r = pick(jobs.r, cur.job), d_out = pick(jobs.d_out, cur.job);
+    const int rows_per_item = pick(jobs.rows_per_item, cur.job);
+    const float* __restrict__ h = pick(jobs.h, cur.job);
+    const float* __restrict__ y0 = pick(jobs.y0, cur.job);
+    __nv_bfloat16* __restrict__ y = pick(jobs.y, cur.job);
+    const int jb = cur.sub, tiles_per_item = rows_per_item >> 4;
+    const __nv_bfloat16* Bs = pick(jobs.B, cur.job) + (size_t)cur.slot * (size_t)d_out * (size_t)r;
     for (int tc = 0; tc < cur.n; tc += 8) {
       // token operand (MMA "B" fragment): column g = token tc+g, k slots <- rho 32p + 8t .. +7
       const bool vx = (tc + g) < cur.n;
@@ -223,29 +263,32 @@ static int stream_grid(long max_items, int n_sms, int ctas_per_sm) {
   return g < 1 ? 1 : (int)g;
 }
 
-cudaError_t launch_lora_shrink_stream(const PlanView& pv, const int* slot_of_expert, const __nv_bfloat16* x,
-                                      const __nv_bfloat16* A, float* h, int r, int d_in, int n_sms,
-                                      cudaStream_t stream) {
-  const int MG = (r + 15) / 16;
-  lora_shrink_stream_kernel<<<stream_grid((long)pv.Smax * MG, n_sms, 8), kShrinkThreads, 0, stream>>>(
-      pv.header, pv.perm, pv.seg_expert, pv.seg_start, slot_of_expert, x, A, h, r, d_in);
+cudaError_t launch_lora_shrink_stream(const PlanView& pv, ShrinkJobs jobs, int n_sms, cudaStream_t stream) {
+  long items = 0;
+  for (int j = 0; j < jobs.n; ++j) {
+    jobs.per_seg[j] = (jobs.r[j] + 15) / 16;
+    items += (long)pv.Smax * jobs.per_seg[j];
+  }
+  lora_shrink_stream_kernel<<<stream_grid(items, n_sms, 8), kShrinkThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab,
+                                                                                       jobs);
   return cudaGetLastError();
 }
 
-cudaError_t launch_lora_expand_stream(const PlanView& pv, const int* slot_of_expert, const float* h,
-                                      const __nv_bfloat16* B, const float* y0, __nv_bfloat16* y, float scale, int r,
-                                      int d_out, int n_sms, cudaStream_t stream) {
-  const int rows_per_item = d_out <= 512 ? 128 : 512;
-  const int JB = (d_out + rows_per_item - 1) / rows_per_item;
-  const int grid = stream_grid((long)pv.Smax * JB, n_sms, 16);
-  if (r <= 32)
-    lora_expand_stream_kernel<1><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_expert, pv.seg_start,
-                                                                      slot_of_expert, h, B, y0, y, scale, r, d_out,
-                                                                      rows_per_item);
+cudaError_t launch_lora_expand_stream(const PlanView& pv, ExpandJobs jobs, float scale, int n_sms,
+                                      cudaStream_t stream) {
+  long items = 0;
+  int rmax = 0;
+  for (int j = 0; j < jobs.n; ++j) {
+    jobs.rows_per_item[j] = jobs.d_out[j] <= 512 ? 128 : 512;
+    jobs.per_seg[j] = (jobs.d_out[j] + jobs.rows_per_item[j] - 1) / jobs.rows_per_item[j];
+    items += (long)pv.Smax * jobs.per_seg[j];
+    rmax = jobs.r[j] > rmax ? jobs.r[j] : rmax;
+  }
+  const int grid = stream_grid(items, n_sms, 16);
+  if (rmax <= 32)
+    lora_expand_stream_kernel<1><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale);
   else
-    lora_expand_stream_kernel<2><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_expert, pv.seg_start,
-                                                                      slot_of_expert, h, B, y0, y, scale, r, d_out,
-                                                                      rows_per_item);
+    lora_expand_stream_kernel<2><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale);
   return cudaGetLastError();
 }
 

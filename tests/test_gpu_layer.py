@@ -123,6 +123,33 @@ def test_request_permutation_and_determinism(mode, stream_impl):
     assert torch.equal(y3, y1[torch.from_numpy(rows).to(DEV)])
 
 
+@pytest.mark.parametrize("mode", MODES)
+def test_grouped_projections_equal_single_calls(mode):
+    # {q,k,v}-like group: shared plan, different shapes; the group's outputs are bit-identical to one call per
+    # projection, and match the oracle.
+    rng = mi.np_rng(13, 1)
+    E, T = 40, 200
+    te = rng.integers(-1, E, size=T).astype(np.int32) if mode == moin.PLAN_SEGMENTS else \
+        np.repeat(rng.integers(0, E, size=2), [130, 70]).astype(np.int32)
+    shapes = [(512, 512, 32), (512, 64, 32), (512, 72, 16), (256, 1024, 64)]
+    plan = moin.plan_build(torch.from_numpy(te).to(DEV), E, mode)
+    cases, jobs, singles = [], [], []
+    for i, (d_in, d_out, r) in enumerate(shapes):
+        pool = mi.make_pool(E, r, d_in, d_out, 13, 10 + i, missing=(3,))
+        case = mi.layer_case(f"g{i}", T, d_in, d_out, pool, te, 2.0, 13, 20 + i)
+        gp = gpu_pool(pool)
+        x, W = case.x.to(DEV), case.W.to(DEV)
+        y = torch.empty(T, d_out, dtype=torch.bfloat16, device=DEV)
+        cases.append(case)
+        jobs.append((x, W, gp, y))
+        singles.append(moin.lora_linear(plan, x, W, gp, 2.0).clone())
+    moin.lora_linear_group(plan, moin.JobGroup(jobs), 2.0)
+    torch.cuda.synchronize()
+    for case, (x, W, gp, y), y1 in zip(cases, jobs, singles):
+        assert torch.equal(y, y1), case.name
+        assert_layer_close(y, oracle_layer(case), case.name)
+
+
 def test_empty_batch_and_argument_errors():
     pool = gpu_pool(mi.make_pool(4, 8, 64, 64, 10, 1))
     x = torch.zeros(0, 64, dtype=torch.bfloat16, device=DEV)
