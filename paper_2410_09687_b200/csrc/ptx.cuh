@@ -104,4 +104,18 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
   return v;
 }
 
+// Optional in-kernel timeline for tuning (compile with -DMOIN_TRACE): MOIN_TSTAMP(e) stores the global timer
+// of event e for this CTA (first writer wins until the trace is reset).  One trace array per translation
+// unit; a unit that wants it read back defines an extern "C" reader (see tc_gemm.cu).
+#ifdef MOIN_TRACE
+static __device__ unsigned long long g_trace[16][256];
+#define MOIN_TSTAMP(e)                                                                         \
+  do {                                                                                         \
+    if ((threadIdx.x & 31) == 0 && blockIdx.x < 256)                                           \
+      atomicCAS(&g_trace[(e)][blockIdx.x], 0ull, global_ns());                                 \
+  } while (0)
+#else
+#define MOIN_TSTAMP(e) do { } while (0)
+#endif
+
 }  // namespace moin

@@ -329,6 +329,16 @@ static int pick_bn(long tiles_m, int N, int n_sms) {
   }
   return 64;
 }
+// Few row tiles (decode): a CTA is bound by the bytes it pulls through its SM's L2 -> shared-memory port,
+// (128 + BN) * K * 2.  This GEMM runs beside the adapter-streaming kernels, so prefer the widest tile (fewest
+// CTAs, least re-reading of x) whose per-CTA bytes stay under a budget that keeps it shorter than the stream.
+static int pick_bn_small_m(int N, int K) {
+  const double budget = 2.2e6;
+  for (int bn : {256, 128}) {
+    if ((128.0 + bn) * K * 2 <= budget && N >= bn) return bn;
+  }
+  return 64;
+}
 
 bool tc_gemm_supported(int T, int d_in, int d_out) { return T >= 1 && d_in >= 64 && (d_in % 8) == 0 && (d_out % 8) == 0; }
 bool tc_router_supported(int Q, int K, int D) { return Q >= 1 && K >= 1 && D >= 64 && (D % 8) == 0; }
@@ -337,7 +347,7 @@ bool tc_fused_supported(int r) { return r >= 8 && r <= 64 && (r % 8) == 0; }
 moin_status launch_tc_gemm(HostState* hs, const __nv_bfloat16* x, const __nv_bfloat16* W, __nv_bfloat16* y, float* y0,
                            int T, int d_in, int d_out, cudaStream_t stream) {
   const long tiles_m = (T + kBM - 1) / kBM;
-  const int bn = pick_bn(tiles_m, d_out, hs->n_sms);
+  const int bn = (tiles_m <= 2 && y0 != nullptr) ? pick_bn_small_m(d_out, d_in) : pick_bn(tiles_m, d_out, hs->n_sms);
   CUtensorMap a, b;
   moin_status st = make_map(&a, x, T, d_in, kBM);
   if (!st) st = make_map(&b, W, d_out, d_in, bn);
