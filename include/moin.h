@@ -252,7 +252,9 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
  * 1/sqrt(head_dim); query head h reads kv head h / (n_heads / n_kv_heads);
  * down(silu(gate(v)) * up(v)); no biases; untied lm_head; no adapter on embedding / lm_head.
  * Storage: residual stream fp32; norm outputs, projection outputs, rotated q/k, attention
- * output, SwiGLU output and logits bf16.  head_dim must be 64.
+ * output, SwiGLU output and logits bf16; the un-normalised attention weights exp(s - max) enter the
+ * P V product as bf16 tensor-core operands (their sum, the softmax normaliser, is taken before rounding).
+ * head_dim must be 64.
  * ------------------------------------------------------------------------------------- */
 typedef struct {
   int32_t n_layers, hidden, n_heads, n_kv_heads, head_dim, ffn, vocab;

@@ -209,7 +209,9 @@ int moin_oracle_lora_linear(const void* x, const void* W, const void* A, const v
  *
  * round_storage != 0 rounds to bf16 wherever the GPU library stores a tensor in bf16
  * (norm outputs, projection outputs, rotated q/k, attention output, SwiGLU output,
- * logits); the residual stream stays unrounded (the library keeps it in fp32).
+ * logits) and where it documents a bf16 tensor-core operand that is never stored (the
+ * un-normalised attention weights exp(s - max)); the residual stream stays unrounded (the
+ * library keeps it in fp32).
  * ------------------------------------------------------------------------------------ */
 typedef struct {
   int32_t n_layers, hidden, n_heads, n_kv_heads, head_dim, ffn, vocab, E, r, n_slots;
@@ -306,7 +308,10 @@ static int run_blocks(const moin_oracle_model* m, int layer_begin, int layer_end
         double den = 0.0;
         for (int64_t u = 0; u <= t; ++u) {
           prob[u] = exp(prob[u] - mx);
-          den += prob[u];
+          den += prob[u];                          /* normaliser: sum of the unrounded weights */
+          prob[u] = maybe_round(prob[u], rnd);     /* storage-rounded variant: the library feeds the weights to the
+                                                      tensor cores as bf16 (the one operand rounding that is not a
+                                                      stored tensor); the exact variant keeps them in double */
         }
         double* ov = att + ((size_t)t * nh + hq) * hd;
         for (int i = 0; i < hd; ++i) {

@@ -350,7 +350,7 @@ size_t moin_lora_linear_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, 
   const size_t parts = (size_t)lora_stream_parts(d_in > 0 ? d_in : 64);
   size_t seg = align_up(parts * (size_t)T * (size_t)(r > 0 ? r : 8) * sizeof(float), 256) +
                align_up((size_t)T * (size_t)d_out * sizeof(float), 256);
-  size_t tiles = align_up(Tp * (size_t)64 * sizeof(__nv_bfloat16), 256);
+  size_t tiles = align_up(2 * Tp * (size_t)64 * sizeof(__nv_bfloat16), 256);   // hi and lo parts of s * (x A^T)
   return (seg > tiles ? seg : tiles) + 256;
 }
 

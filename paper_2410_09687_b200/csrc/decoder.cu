@@ -271,13 +271,11 @@ static DecoderWorkspace carve(const moin_model* m, int R, int T, int max_seqlen,
   w.plan_bytes = moin_plan_bytes(T, m->E > 0 ? m->E : 1);
   w.plan = take(w.plan_bytes);
   size_t lb = 0;
-  const size_t dims[4][2] = {{H, qd}, {H, F}, {F, H}, {H, (size_t)m->vocab}};
   int r = 8;
   if (m->pools) r = m->pools[0].r;
-  for (auto& d : dims) {
-    size_t b = moin_lora_linear_workspace_bytes(T, (int)d[0], (int)d[1], r);
-    lb = b > lb ? b : lb;
-  }
+  auto one = [&](size_t din, size_t dout) { return moin_lora_linear_workspace_bytes(T, (int)din, (int)dout, r); };
+  const size_t groups[5] = {one(H, qd) + 2 * one(H, kvd), one(qd, H), 2 * one(H, F), one(F, H), one(H, (size_t)m->vocab)};
+  for (size_t b : groups) lb = b > lb ? b : lb;
   w.lora_bytes = lb;
   w.lora = take(lb);
   w.total = off;
@@ -342,14 +340,30 @@ extern "C" moin_status moin_decoder_forward(const moin_model* m, const int32_t* 
     return moin_lora_linear(lora ? &plan : nullptr, in, m->W[layer * 7 + p], lora ? &m->pools[layer * 7 + p] : nullptr,
                             m->lora_scale, T, d_in, d_out, out, w.lora, w.lora_bytes, stream);
   };
+  // projections of a block that read the same input and do not depend on one another go out as one group
+  auto proj_group = [&](int layer, int p0, int n, const void* in, const int* d_in, const int* d_out,
+                        void* const* outs) -> moin_status {
+    if (!lora) {
+      for (int i = 0; i < n; ++i) {
+        moin_status e = proj(layer, p0 + i, in, d_in[i], d_out[i], outs[i]);
+        if (e) return e;
+      }
+      return MOIN_OK;
+    }
+    moin_lora_job jobs[MOIN_MAX_GROUP];
+    for (int i = 0; i < n; ++i) jobs[i] = {in, m->W[layer * 7 + p0 + i], &m->pools[layer * 7 + p0 + i], outs[i]};
+    return moin_lora_linear_group(&plan, jobs, n, m->lora_scale, w.lora, w.lora_bytes, stream);
+  };
   const float scale_log2 = 1.4426950408889634f / sqrtf(64.f);
   const __nv_bfloat16* pending = nullptr;
   for (int l = lb; l < le; ++l) {
     { ProfScope prof(MOIN_K_GLUE, 1, s);
       add_rmsnorm_kernel<<<T, 256, 0, s>>>(w.res, pending, (const __nv_bfloat16*)m->attn_norm[l], w.xn, H, m->rms_eps, nullptr); }
-    if ((st = proj(l, 0, w.xn, H, qd, w.q))) return st;
-    if ((st = proj(l, 1, w.xn, H, kvd, w.k))) return st;
-    if ((st = proj(l, 2, w.xn, H, kvd, w.v))) return st;
+    {
+      const int din[3] = {H, H, H}, dout[3] = {qd, kvd, kvd};
+      void* const outs[3] = {w.q, w.k, w.v};
+      if ((st = proj_group(l, 0, 3, w.xn, din, dout, outs))) return st;
+    }
     { ProfScope prof(MOIN_K_GLUE, 2, s);
       rope_kernel<<<(int)(((long)T * nh * 32 + 255) / 256), 256, 0, s>>>(w.q, w.pos, w.rope, T, nh);
       rope_kernel<<<(int)(((long)T * nkv * 32 + 255) / 256), 256, 0, s>>>(w.k, w.pos, w.rope, T, nkv); }
@@ -358,8 +372,11 @@ extern "C" moin_status moin_decoder_forward(const moin_model* m, const int32_t* 
     if ((st = proj(l, 3, w.att, qd, H, w.o))) return st;
     { ProfScope prof(MOIN_K_GLUE, 1, s);
       add_rmsnorm_kernel<<<T, 256, 0, s>>>(w.res, w.o, (const __nv_bfloat16*)m->mlp_norm[l], w.xn, H, m->rms_eps, nullptr); }
-    if ((st = proj(l, 4, w.xn, H, F, w.gate))) return st;
-    if ((st = proj(l, 5, w.xn, H, F, w.up))) return st;
+    {
+      const int din[2] = {H, H}, dout[2] = {F, F};
+      void* const outs[2] = {w.gate, w.up};
+      if ((st = proj_group(l, 4, 2, w.xn, din, dout, outs))) return st;
+    }
     { ProfScope prof(MOIN_K_GLUE, 1, s);
       swiglu_kernel<<<(int)(((long)T * F / 8 + 255) / 256), 256, 0, s>>>(w.gate, w.up, (long)T * F / 8); }
     if ((st = proj(l, 6, w.gate, F, H, w.o))) return st;

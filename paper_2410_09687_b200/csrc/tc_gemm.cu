@@ -11,13 +11,13 @@
 //              EPI_ROUTER  running (max, argmax) of acc * inv_norm[col], merged across tiles with a
 //                          64-bit atomicMax on (orderable(sim) << 32 | ~col): order independent,
 //                          lowest index wins ties
-//              EPI_SHRINK  hb = bf16(scale * acc) for the LoRA rank columns
+//              EPI_SHRINK  scale * acc for the LoRA rank columns, stored as bf16 hi + lo parts
 // Two accumulator buffers in TMEM let the epilogue of tile i overlap the MMAs of tile i+1.
 //
 // Row tiles come either from a regular grid over M or from a batch plan (runs of tokens with
-// one expert, <= 128 rows).  With a plan, EPI_STORE appends one extra K block per tile taken
-// from hb[rows, r] and B_e[d_out, r] of the tile's adapter: y = [x | s h] [W ; B_e]^T, so
-// the low-rank term is added inside the accumulator and y is written once.
+// one expert, <= 128 rows).  With a plan, EPI_STORE appends two extra K blocks per tile taken
+// from hi/lo[rows, r] and B_e[d_out, r] of the tile's adapter: y = [x | hi(s h) | lo(s h)] [W ; B_e ; B_e]^T,
+// so the low-rank term is added inside the accumulator (to ~fp32 accuracy) and y is written once.
 // Every wait on an mbarrier is bounded; on expiry the kernel raises the status flag and returns.
 #include <cuda.h>
 
@@ -41,6 +41,7 @@ struct TcParams {
   int tail_r;                  // EPI_STORE with plan: LoRA rank of the appended K block (0 = none)
   int rows_per_slot;           // rows of the B-side pool tensor per adapter slot (d_out, or r for EPI_SHRINK)
   __nv_bfloat16* y;            // EPI_STORE / EPI_SHRINK output, leading dimension ldy
+  __nv_bfloat16* y_lo;         // EPI_SHRINK: low part, value - bf16(value), same layout as y
   float* y0;                   // EPI_STORE: optional fp32 copy
   int ldy;
   float scale;                 // EPI_SHRINK
@@ -81,7 +82,8 @@ template <int BN> struct TcCfg {
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
+               const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmA3,
+               const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
   using Cfg = TcCfg<BN>;
   constexpr int S = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
@@ -145,7 +147,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int row0, rows, n0, slot;
         tile_info(tile, row0, rows, n0, slot);
         const bool tail = (EPI == EPI_STORE) && planned && p.tail_r > 0 && slot >= 0;
-        const int nkb = nkb_main + (tail ? 1 : 0);
+        const int nkb = nkb_main + (tail ? 2 : 0);   // tail: [hi(s h) | lo(s h)] x [B_e ; B_e]
         const int brow = (EPI == EPI_SHRINK) ? (slot >= 0 ? slot : 0) * p.rows_per_slot : n0;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const uint32_t s = it % S, ph = (it / S) & 1u;
@@ -156,7 +158,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tma_load_2d(sa, &tmA, full0 + 8 * s, kb * kBK, row0);
             tma_load_2d(sb, &tmB, full0 + 8 * s, kb * kBK, brow);
           } else {
-            tma_load_2d(sa, &tmA2, full0 + 8 * s, 0, row0);
+            tma_load_2d(sa, kb == nkb_main ? &tmA2 : &tmA3, full0 + 8 * s, 0, row0);
             tma_load_2d(sb, &tmB2, full0 + 8 * s, 0, slot * p.rows_per_slot + n0);
           }
         }
@@ -172,7 +174,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int row0, rows, n0, slot;
         tile_info(tile, row0, rows, n0, slot);
         const bool tail = (EPI == EPI_STORE) && planned && p.tail_r > 0 && slot >= 0;
-        const int nkb = nkb_main + (tail ? 1 : 0);
+        const int nkb = nkb_main + (tail ? 2 : 0);
         const uint32_t acc = lt & 1u, aph = (lt >> 1) & 1u;
         if (!(ok = mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag, p.status, 2))) break;
         tc_fence_after();
@@ -233,12 +235,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
             if (n0 + c + j < p.N) {  // N is a multiple of 8
+              float f[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]) * sc;
               uint4 o;
-              o.x = pack_bf16(__uint_as_float(v[j + 0]) * sc, __uint_as_float(v[j + 1]) * sc);
-              o.y = pack_bf16(__uint_as_float(v[j + 2]) * sc, __uint_as_float(v[j + 3]) * sc);
-              o.z = pack_bf16(__uint_as_float(v[j + 4]) * sc, __uint_as_float(v[j + 5]) * sc);
-              o.w = pack_bf16(__uint_as_float(v[j + 6]) * sc, __uint_as_float(v[j + 7]) * sc);
+              o.x = pack_bf16(f[0], f[1]);
+              o.y = pack_bf16(f[2], f[3]);
+              o.z = pack_bf16(f[4], f[5]);
+              o.w = pack_bf16(f[6], f[7]);
               *reinterpret_cast<uint4*>(yrow + j) = o;
+              if (EPI == EPI_SHRINK) {   // low part, so that hi + lo carries the value to ~fp32 accuracy
+                uint4 l;
+                l.x = pack_bf16(f[0] - bf16_lo(o.x), f[1] - bf16_hi(o.x));
+                l.y = pack_bf16(f[2] - bf16_lo(o.y), f[3] - bf16_hi(o.y));
+                l.z = pack_bf16(f[4] - bf16_lo(o.z), f[5] - bf16_hi(o.z));
+                l.w = pack_bf16(f[6] - bf16_lo(o.w), f[7] - bf16_hi(o.w));
+                *reinterpret_cast<uint4*>(p.y_lo + grow * (size_t)p.ldy + n0 + c + j) = l;
+              }
               if (EPI == EPI_STORE && p.y0) {
                 float* y0row = p.y0 + grow * (size_t)p.ldy + n0 + c + j;
                 *reinterpret_cast<uint4*>(y0row) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -308,7 +321,8 @@ moin_status make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t
 
 template <int BN, int EPI>
 static moin_status launch_cfg(HostState* hs, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& a2,
-                              const CUtensorMap& b2, const TcParams& p, long max_tiles, cudaStream_t stream) {
+                              const CUtensorMap& a3, const CUtensorMap& b2, const TcParams& p, long max_tiles,
+                              cudaStream_t stream) {
   using Cfg = TcCfg<BN>;
   static bool configured = false;
   if (!configured) {
@@ -319,7 +333,7 @@ static moin_status launch_cfg(HostState* hs, const CUtensorMap& a, const CUtenso
   }
   long grid = max_tiles < hs->n_sms ? max_tiles : hs->n_sms;
   if (grid < 1) grid = 1;
-  tc_gemm_kernel<BN, EPI><<<(int)grid, kTcThreads, Cfg::kSmemBytes, stream>>>(a, b, a2, b2, p);
+  tc_gemm_kernel<BN, EPI><<<(int)grid, kTcThreads, Cfg::kSmemBytes, stream>>>(a, b, a2, a3, b2, p);
   return record_cuda(cudaGetLastError());
 }
 
@@ -355,9 +369,9 @@ moin_status launch_tc_gemm(HostState* hs, const __nv_bfloat16* x, const __nv_bfl
   TcParams p = {};
   p.M = T; p.N = d_out; p.K = d_in; p.y = y; p.y0 = y0; p.ldy = d_out; p.scale = 1.f; p.status = hs->status;
   const long tiles = tiles_m * ((d_out + bn - 1) / bn);
-  if (bn == 256) return launch_cfg<256, EPI_STORE>(hs, a, b, a, b, p, tiles, stream);
-  if (bn == 128) return launch_cfg<128, EPI_STORE>(hs, a, b, a, b, p, tiles, stream);
-  return launch_cfg<64, EPI_STORE>(hs, a, b, a, b, p, tiles, stream);
+  if (bn == 256) return launch_cfg<256, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream);
+  if (bn == 128) return launch_cfg<128, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream);
+  return launch_cfg<64, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream);
 }
 
 moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
@@ -371,9 +385,9 @@ moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_b
   TcParams p = {};
   p.M = Q; p.N = K; p.K = D; p.inv_norm = inv_norm; p.keys = keys; p.status = hs->status;
   const long tiles = tiles_m * ((K + bn - 1) / bn);
-  if (bn == 256) return launch_cfg<256, EPI_ROUTER>(hs, a, b, a, b, p, tiles, stream);
-  if (bn == 128) return launch_cfg<128, EPI_ROUTER>(hs, a, b, a, b, p, tiles, stream);
-  return launch_cfg<64, EPI_ROUTER>(hs, a, b, a, b, p, tiles, stream);
+  if (bn == 256) return launch_cfg<256, EPI_ROUTER>(hs, a, b, a, a, b, p, tiles, stream);
+  if (bn == 128) return launch_cfg<128, EPI_ROUTER>(hs, a, b, a, a, b, p, tiles, stream);
+  return launch_cfg<64, EPI_ROUTER>(hs, a, b, a, a, b, p, tiles, stream);
 }
 
 moin_status launch_tc_lora_tiles(HostState* hs, const PlanView& pv, const moin_pool* pool, const __nv_bfloat16* x,
@@ -382,10 +396,12 @@ moin_status launch_tc_lora_tiles(HostState* hs, const PlanView& pv, const moin_p
   const int T = pv.T, d_in = pool->d_in, d_out = pool->d_out, r = pool->r;
   // upper bound on row tiles without reading the plan back: every run adds at most one partial tile
   const long max_tiles_m = T;  // grid is capped at the SM count; the kernel reads the true count
-  CUtensorMap ax, bA, bW, ah, bB;
+  CUtensorMap ax, bA, bW, ah, al, bB;
+  __nv_bfloat16* hb_lo = hb + (size_t)T * r;   // low parts follow the high parts in the workspace
   moin_status st = make_map(&ax, x, T, d_in, kBM);
   if (!st) st = make_map(&bA, pool->A, (uint64_t)pool->n_slots * r, d_in, 64);
   if (!st) st = make_map(&ah, hb, T, r, kBM);
+  if (!st) st = make_map(&al, hb_lo, T, r, kBM);
   if (!st) st = make_map(&bB, pool->B, (uint64_t)pool->n_slots * d_out, r, 256);
   if (st) return st;
   // 1. hb[row, :r] = bf16(scale * x A_e^T)   (one N tile of 64 columns, rank columns stored)
@@ -393,9 +409,9 @@ moin_status launch_tc_lora_tiles(HostState* hs, const PlanView& pv, const moin_p
     ProfScope prof(MOIN_K_SHRINK_TC, 1, stream);
     TcParams p = {};
     p.M = T; p.N = r; p.K = d_in; p.header = pv.header; p.tile_row0 = pv.tile_row0; p.tile_rows = pv.tile_rows;
-    p.tile_expert = pv.tile_expert; p.slot_of_expert = pool->slot_of_expert; p.rows_per_slot = r; p.y = hb; p.ldy = r;
+    p.tile_expert = pv.tile_expert; p.slot_of_expert = pool->slot_of_expert; p.rows_per_slot = r; p.y = hb; p.y_lo = hb_lo; p.ldy = r;
     p.scale = scale; p.status = hs->status;
-    st = launch_cfg<64, EPI_SHRINK>(hs, ax, bA, ax, bA, p, max_tiles_m, stream);
+    st = launch_cfg<64, EPI_SHRINK>(hs, ax, bA, ax, ax, bA, p, max_tiles_m, stream);
     if (st) return st;
   }
   // 2. y = [x | hb] [W ; B_e]^T
@@ -410,9 +426,9 @@ moin_status launch_tc_lora_tiles(HostState* hs, const PlanView& pv, const moin_p
   p.tile_expert = pv.tile_expert; p.slot_of_expert = pool->slot_of_expert; p.tail_r = r; p.rows_per_slot = d_out;
   p.y = y; p.ldy = d_out; p.scale = 1.f; p.status = hs->status;
   const long tiles = max_tiles_m * ((d_out + bn - 1) / bn);
-  if (bn == 256) return launch_cfg<256, EPI_STORE>(hs, ax, bW, ah, bB, p, tiles, stream);
-  if (bn == 128) return launch_cfg<128, EPI_STORE>(hs, ax, bW, ah, bB, p, tiles, stream);
-  return launch_cfg<64, EPI_STORE>(hs, ax, bW, ah, bB, p, tiles, stream);
+  if (bn == 256) return launch_cfg<256, EPI_STORE>(hs, ax, bW, ah, al, bB, p, tiles, stream);
+  if (bn == 128) return launch_cfg<128, EPI_STORE>(hs, ax, bW, ah, al, bB, p, tiles, stream);
+  return launch_cfg<64, EPI_STORE>(hs, ax, bW, ah, al, bB, p, tiles, stream);
 }
 
 }  // namespace moin
