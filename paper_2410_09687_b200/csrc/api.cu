@@ -444,9 +444,17 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
   float* h[kMaxStreamJobs];
   float* y0[kMaxStreamJobs];
   int parts[kMaxStreamJobs];
-  const bool tma_stream = hs->stream_impl == 2 && n_jobs == 1;   // MOIN_OPT_STREAM_IMPL: TMA-staged kernels (one job)
+  bool tma_stream = hs->stream_impl == 2;   // MOIN_OPT_STREAM_IMPL: TMA-staged kernels
+  for (int j = 0; j < n_jobs; ++j) tma_stream = tma_stream && lora_shrink_tma_supported(d_in[j]);
+  int* queue = reinterpret_cast<int*>(ws_job[0] + moin_lora_linear_workspace_bytes(T, d_in[0], d_out[0], r[0]) - 256);
+  const moin_pool* pools[kMaxStreamJobs];
+  const __nv_bfloat16* xs[kMaxStreamJobs];
+  __nv_bfloat16* ys[kMaxStreamJobs];
   for (int j = 0; j < n_jobs; ++j) {
-    parts[j] = (tma_stream && lora_shrink_tma_supported(d_in[j])) ? lora_stream_parts(d_in[j]) : 1;
+    pools[j] = jobs[j].pool;
+    xs[j] = (const __nv_bfloat16*)jobs[j].x;
+    ys[j] = (__nv_bfloat16*)jobs[j].y;
+    parts[j] = tma_stream ? lora_stream_parts(d_in[j]) : 1;
     h[j] = reinterpret_cast<float*>(ws_job[j]);   // [parts][T][r] (partial) shrink results
     y0[j] = reinterpret_cast<float*>(ws_job[j] + align_up((size_t)lora_stream_parts(d_in[j]) * (size_t)T * (size_t)r[j] * sizeof(float), 256));
   }
@@ -469,8 +477,8 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
   moin_status st_shrink;
   {
     ProfScope prof(MOIN_K_SHRINK_STREAM, 1, s);
-    if (tma_stream && parts[0] >= 1 && lora_shrink_tma_supported(d_in[0])) {
-      st_shrink = launch_lora_shrink_tma(hs, pv, jobs[0].pool, (const __nv_bfloat16*)jobs[0].x, h[0], s);
+    if (tma_stream) {
+      st_shrink = launch_lora_shrink_tma(hs, pv, pools, xs, h, n_jobs, queue, lora_stream_ring_bytes(), s);
     } else {
       ShrinkJobs sj = {};
       sj.n = n_jobs;
@@ -494,7 +502,8 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
   if (st_gemm) return st_gemm;
   if (st_shrink) return st_shrink;
   ProfScope prof(MOIN_K_EXPAND_STREAM, 1, s);
-  if (tma_stream) return launch_lora_expand_tma(hs, pv, jobs[0].pool, h[0], parts[0], y0[0], (__nv_bfloat16*)jobs[0].y, scale, s);
+  if (tma_stream)
+    return launch_lora_expand_tma(hs, pv, pools, h, parts, y0, ys, n_jobs, scale, queue, lora_stream_ring_bytes(), s);
   ExpandJobs ej = {};
   ej.n = n_jobs;
   for (int j = 0; j < n_jobs; ++j) {

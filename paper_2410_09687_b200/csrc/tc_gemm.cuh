@@ -27,13 +27,18 @@ moin_status launch_tc_lora_tiles(HostState* hs, const PlanView& pv, const moin_p
                                  const __nv_bfloat16* W, __nv_bfloat16* y, __nv_bfloat16* hb, float scale,
                                  cudaStream_t stream);
 
-// TMA-staged segmented LoRA kernels (short segments).  The shrink writes lora_stream_parts(d_in) partial
-// results hpart[part][T][r]; the expand sums them in a fixed order.
+// TMA-staged segmented LoRA kernels (short segments), up to 4 projections per launch.  The shrink writes
+// lora_stream_parts(d_in) partial results hpart[part][T][r] per projection; the expand sums them in index order.
+// `queue` is one int of device scratch (the work counter, reset by the launcher on `stream`).
 int lora_stream_parts(int d_in);
 bool lora_shrink_tma_supported(int d_in);
-moin_status launch_lora_shrink_tma(HostState* hs, const PlanView& pv, const moin_pool* pool, const __nv_bfloat16* x,
-                                   float* hpart, cudaStream_t stream);
-moin_status launch_lora_expand_tma(HostState* hs, const PlanView& pv, const moin_pool* pool, const float* hpart, int KP,
-                                   const float* y0, __nv_bfloat16* y, float scale, cudaStream_t stream);
+size_t lora_stream_ring_bytes();
+moin_status launch_lora_shrink_tma(HostState* hs, const PlanView& pv, const moin_pool* const* pools,
+                                   const __nv_bfloat16* const* x, float* const* hpart, int n_jobs, int* queue,
+                                   size_t ring_bytes, cudaStream_t stream);
+moin_status launch_lora_expand_tma(HostState* hs, const PlanView& pv, const moin_pool* const* pools,
+                                   const float* const* hpart, const int* parts, const float* const* y0,
+                                   __nv_bfloat16* const* y, int n_jobs, float scale, int* queue, size_t ring_bytes,
+                                   cudaStream_t stream);
 
 }  // namespace moin

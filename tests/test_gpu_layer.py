@@ -124,7 +124,7 @@ def test_request_permutation_and_determinism(mode, stream_impl):
 
 
 @pytest.mark.parametrize("mode", MODES)
-def test_grouped_projections_equal_single_calls(mode):
+def test_grouped_projections_equal_single_calls(mode, stream_impl):
     # {q,k,v}-like group: shared plan, different shapes; the group's outputs are bit-identical to one call per
     # projection, and match the oracle.
     rng = mi.np_rng(13, 1)
