@@ -154,106 +154,134 @@ lora_shrink_stream_kernel(const int* __restrict__ header, const int* __restrict_
 
 // y[perm[pos]][j] = bf16( y0[perm[pos]][j] + scale * sum_rho B[slot][j][rho] * h[pos][rho] )
 // h is split into bf16 hi + lo parts (two MMAs) so the low-rank term keeps ~fp32 accuracy.
-// Work item = (job, segment, block of rows_per_item output features); each warp walks its 16-row tiles
-// kExpandTilesPerBatch at a time with the adapter rows and the base values y0 loaded together.
+//
+// The unit of work is one 16-row tile of B for one (segment, job); units are ordered (segment, job, tile)
+// and every warp of the grid takes one contiguous, equally long range of them (tiles need no reduction
+// across each other, so a range may start and end anywhere).  All warps therefore stream the same number
+// of adapter bytes, whatever the mix of projection widths in the launch, and a warp's range is contiguous
+// in memory inside a (segment, job).  A warp walks its range kExpandTilesPerBatch tiles at a time with
+// the adapter rows and the base values y0 of a batch loaded together.  `jobs.per_seg[j]` = tiles of job j.
 template <int P>  // number of 32-wide rho groups: ceil(max r / 32)
 __global__ void __launch_bounds__(kExpandThreads, 4)
 lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict__ perm,
-                          const int4* __restrict__ seg_tab, const ExpandJobs jobs, float scale) {
+                          const int4* __restrict__ seg_tab, const ExpandJobs jobs, float scale, int tps) {
   constexpr int TB = kExpandTilesPerBatch;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int nseg = header[PH_NSEG];
-  int items = 0;
+  const long long wid = (long long)blockIdx.x * (kExpandThreads / 32) + warp;
+  const long long nw = (long long)gridDim.x * (kExpandThreads / 32);
+  const int nseg = __ldg(header + PH_NSEG);
+  const long long units = (long long)nseg * tps;
+  long long u = units * wid / nw;
+  const long long u_end = units * (wid + 1) / nw;
+  while (u < u_end) {
+    // ---- segment: expert, rows, adapter slots of all jobs (one hop after the table entry)
+    const int seg = (int)(u / tps);
+    const int4 e = __ldg(seg_tab + seg);   // (expert, start, length, -)
+    const int s0 = e.y, n = e.z;
+    int slots[kMaxStreamJobs];
 #pragma unroll
-  for (int j = 0; j < kMaxStreamJobs; ++j)
-    if (j < jobs.n) items += nseg * jobs.per_seg[j];
-  int item = blockIdx.x;
-  SegMeta nxt = load_seg(seg_tab, jobs, item, items, nseg);
-  for (; item < items; item += gridDim.x) {
-    const SegMeta cur = nxt;
-    nxt = load_seg(seg_tab, jobs, item + gridDim.x, items, nseg);
-    if (cur.slot < 0) continue;
-    const int r = pick(jobs.r, cur.job), d_out = pick(jobs.d_out, cur.job);
-    const int rows_per_item = pick(jobs.rows_per_item, cur.job);
-    const float* __restrict__ h = pick(jobs.h, cur.job);
-    const float* __restrict__ y0 = pick(jobs.y0, cur.job);
-    __nv_bfloat16* __restrict__ y = pick(jobs.y, cur.job);
-    const int jb = cur.sub, tiles_per_item = rows_per_item >> 4;
-    const __nv_bfloat16* Bs = pick(jobs.B, cur.job) + (size_t)cur.slot * (size_t)d_out * (size_t)r;
-    for (int tc = 0; tc < cur.n; tc += 8) {
-      // token operand (MMA "B" fragment): column g = token tc+g, k slots <- rho 32p + 8t .. +7
-      const bool vx = (tc + g) < cur.n;
-      const int my_row = vx ? perm[cur.s0 + tc + g] : -1;
-      uint32_t hh[P][4], hl[P][4];
+    for (int j = 0; j < kMaxStreamJobs; ++j) slots[j] = (j < jobs.n) ? __ldg(jobs.slot_of_expert[j] + e.x) : -1;
+    const int row_first = (g < n) ? __ldg(perm + s0 + g) : -1;
+    const long long seg_end = (long long)(seg + 1) * tps;
+    int rem = (int)(u - (long long)seg * tps);
+    int job = 0;
 #pragma unroll
-      for (int p = 0; p < P; ++p) {
-        const int rb = 32 * p + 8 * t;
-        float v[8];
-        if (vx && rb < r) {
-          const float4 f0 = *reinterpret_cast<const float4*>(h + (size_t)(cur.s0 + tc + g) * r + rb);
-          const float4 f1 = *reinterpret_cast<const float4*>(h + (size_t)(cur.s0 + tc + g) * r + rb + 4);
-          v[0] = f0.x; v[1] = f0.y; v[2] = f0.z; v[3] = f0.w; v[4] = f1.x; v[5] = f1.y; v[6] = f1.z; v[7] = f1.w;
-        } else {
-#pragma unroll
-          for (int q = 0; q < 8; ++q) v[q] = 0.f;
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float s0v = v[2 * q] * scale, s1v = v[2 * q + 1] * scale;
-          const uint32_t hi = pack_bf16(s0v, s1v);
-          hh[p][q] = hi;
-          hl[p][q] = pack_bf16(s0v - bf16_lo(hi), s1v - bf16_hi(hi));
-        }
+    for (int j = 0; j + 1 < kMaxStreamJobs; ++j) {
+      if (job == j && j + 1 < jobs.n && rem >= jobs.per_seg[j]) {
+        rem -= jobs.per_seg[j];
+        job = j + 1;
       }
-      const int row_c0 = __shfl_sync(0xffffffffu, my_row, (2 * t) * 4);
-      const int row_c1 = __shfl_sync(0xffffffffu, my_row, (2 * t + 1) * 4);
-      for (int tb = warp * TB; tb < tiles_per_item; tb += 4 * TB) {
-        uint4 a0[TB][P], a1[TB][P];
-        float b0[TB][4];
-#pragma unroll
-        for (int i = 0; i < TB; ++i) {
-          const int j0 = jb * rows_per_item + (tb + i) * 16;
-          const int ja = j0 + g, jc = j0 + g + 8;
-          const bool va = (tb + i) < tiles_per_item && ja < d_out, vc = (tb + i) < tiles_per_item && jc < d_out;
+    }
+    // ---- (segment, job) pieces of the range
+    while (u < u_end && u < seg_end) {
+      const int tiles_j = pick(jobs.per_seg, job);
+      const int tile0 = rem;
+      const long long left = u_end - u;
+      const int tile1 = (left < (long long)(tiles_j - tile0)) ? tile0 + (int)left : tiles_j;
+      const int slot = pick(slots, job);
+      if (slot >= 0) {
+        const int r = pick(jobs.r, job), d_out = pick(jobs.d_out, job);
+        const float* __restrict__ h = pick(jobs.h, job);
+        const float* __restrict__ y0 = pick(jobs.y0, job);
+        __nv_bfloat16* __restrict__ y = pick(jobs.y, job);
+        const __nv_bfloat16* Bs = pick(jobs.B, job) + (size_t)slot * (size_t)d_out * (size_t)r;
+        for (int tc = 0; tc < n; tc += 8) {
+          // token operand (MMA "B" fragment): column g = token tc+g, k slots <- rho 32p + 8t .. +7
+          const bool vx = (tc + g) < n;
+          const int my_row = (tc == 0) ? row_first : (vx ? __ldg(perm + s0 + tc + g) : -1);
+          uint32_t hh[P][4], hl[P][4];
 #pragma unroll
           for (int p = 0; p < P; ++p) {
             const int rb = 32 * p + 8 * t;
-            const uint4 z = make_uint4(0, 0, 0, 0);
-            a0[i][p] = (va && rb < r) ? ldg_stream(Bs + (size_t)ja * r + rb) : z;
-            a1[i][p] = (vc && rb < r) ? ldg_stream(Bs + (size_t)jc * r + rb) : z;
-          }
-          b0[i][0] = (va && row_c0 >= 0) ? __ldg(y0 + (size_t)row_c0 * d_out + ja) : 0.f;
-          b0[i][1] = (va && row_c1 >= 0) ? __ldg(y0 + (size_t)row_c1 * d_out + ja) : 0.f;
-          b0[i][2] = (vc && row_c0 >= 0) ? __ldg(y0 + (size_t)row_c0 * d_out + jc) : 0.f;
-          b0[i][3] = (vc && row_c1 >= 0) ? __ldg(y0 + (size_t)row_c1 * d_out + jc) : 0.f;
-        }
+            float v[8];
+            if (vx && rb < r) {
+              const float4 f0 = *reinterpret_cast<const float4*>(h + (size_t)(s0 + tc + g) * r + rb);
+              const float4 f1 = *reinterpret_cast<const float4*>(h + (size_t)(s0 + tc + g) * r + rb + 4);
+              v[0] = f0.x; v[1] = f0.y; v[2] = f0.z; v[3] = f0.w; v[4] = f1.x; v[5] = f1.y; v[6] = f1.z; v[7] = f1.w;
+            } else {
 #pragma unroll
-        for (int i = 0; i < TB; ++i) {
-          const int j0 = jb * rows_per_item + (tb + i) * 16;
-          const int ja = j0 + g, jc = j0 + g + 8;
-          const bool va = (tb + i) < tiles_per_item && ja < d_out, vc = (tb + i) < tiles_per_item && jc < d_out;
-          float c[4] = {0.f, 0.f, 0.f, 0.f};
+              for (int q = 0; q < 8; ++q) v[q] = 0.f;
+            }
 #pragma unroll
-          for (int p = 0; p < P; ++p) {
-            mma_bf16_16816(c, a0[i][p].x, a1[i][p].x, a0[i][p].y, a1[i][p].y, hl[p][0], hl[p][1]);
-            mma_bf16_16816(c, a0[i][p].z, a1[i][p].z, a0[i][p].w, a1[i][p].w, hl[p][2], hl[p][3]);
-            mma_bf16_16816(c, a0[i][p].x, a1[i][p].x, a0[i][p].y, a1[i][p].y, hh[p][0], hh[p][1]);
-            mma_bf16_16816(c, a0[i][p].z, a1[i][p].z, a0[i][p].w, a1[i][p].w, hh[p][2], hh[p][3]);
+            for (int q = 0; q < 4; ++q) {
+              const float s0v = v[2 * q] * scale, s1v = v[2 * q + 1] * scale;
+              const uint32_t hi = pack_bf16(s0v, s1v);
+              hh[p][q] = hi;
+              hl[p][q] = pack_bf16(s0v - bf16_lo(hi), s1v - bf16_hi(hi));
+            }
           }
-          // c0:(ja, col 2t) c1:(ja, col 2t+1) c2:(jc, col 2t) c3:(jc, col 2t+1)
-          if (row_c0 >= 0) {
-            const size_t o = (size_t)row_c0 * d_out;
-            if (va) y[o + ja] = __float2bfloat16_rn(b0[i][0] + c[0]);
-            if (vc) y[o + jc] = __float2bfloat16_rn(b0[i][2] + c[2]);
-          }
-          if (row_c1 >= 0) {
-            const size_t o = (size_t)row_c1 * d_out;
-            if (va) y[o + ja] = __float2bfloat16_rn(b0[i][1] + c[1]);
-            if (vc) y[o + jc] = __float2bfloat16_rn(b0[i][3] + c[3]);
+          const int row_c0 = __shfl_sync(0xffffffffu, my_row, (2 * t) * 4);
+          const int row_c1 = __shfl_sync(0xffffffffu, my_row, (2 * t + 1) * 4);
+          for (int tb = tile0; tb < tile1; tb += TB) {
+            uint4 a0[TB][P], a1[TB][P];
+            float b0[TB][4];
+#pragma unroll
+            for (int i = 0; i < TB; ++i) {
+              const int ja = (tb + i) * 16 + g, jc = ja + 8;
+              const bool va = (tb + i) < tile1 && ja < d_out, vc = (tb + i) < tile1 && jc < d_out;
+#pragma unroll
+              for (int p = 0; p < P; ++p) {
+                const int rb = 32 * p + 8 * t;
+                const uint4 z = make_uint4(0, 0, 0, 0);
+                a0[i][p] = (va && rb < r) ? ldg_stream(Bs + (size_t)ja * r + rb) : z;
+                a1[i][p] = (vc && rb < r) ? ldg_stream(Bs + (size_t)jc * r + rb) : z;
+              }
+              b0[i][0] = (va && row_c0 >= 0) ? __ldg(y0 + (size_t)row_c0 * d_out + ja) : 0.f;
+              b0[i][1] = (va && row_c1 >= 0) ? __ldg(y0 + (size_t)row_c1 * d_out + ja) : 0.f;
+              b0[i][2] = (vc && row_c0 >= 0) ? __ldg(y0 + (size_t)row_c0 * d_out + jc) : 0.f;
+              b0[i][3] = (vc && row_c1 >= 0) ? __ldg(y0 + (size_t)row_c1 * d_out + jc) : 0.f;
+            }
+#pragma unroll
+            for (int i = 0; i < TB; ++i) {
+              const int ja = (tb + i) * 16 + g, jc = ja + 8;
+              const bool va = (tb + i) < tile1 && ja < d_out, vc = (tb + i) < tile1 && jc < d_out;
+              float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+              for (int p = 0; p < P; ++p) {
+                mma_bf16_16816(c, a0[i][p].x, a1[i][p].x, a0[i][p].y, a1[i][p].y, hl[p][0], hl[p][1]);
+                mma_bf16_16816(c, a0[i][p].z, a1[i][p].z, a0[i][p].w, a1[i][p].w, hl[p][2], hl[p][3]);
+                mma_bf16_16816(c, a0[i][p].x, a1[i][p].x, a0[i][p].y, a1[i][p].y, hh[p][0], hh[p][1]);
+                mma_bf16_16816(c, a0[i][p].z, a1[i][p].z, a0[i][p].w, a1[i][p].w, hh[p][2], hh[p][3]);
+              }
+              // c0:(ja, col 2t) c1:(ja, col 2t+1) c2:(jc, col 2t) c3:(jc, col 2t+1)
+              if (row_c0 >= 0) {
+                const size_t o = (size_t)row_c0 * d_out;
+                if (va) y[o + ja] = __float2bfloat16_rn(b0[i][0] + c[0]);
+                if (vc) y[o + jc] = __float2bfloat16_rn(b0[i][2] + c[2]);
+              }
+              if (row_c1 >= 0) {
+                const size_t o = (size_t)row_c1 * d_out;
+                if (va) y[o + ja] = __float2bfloat16_rn(b0[i][1] + c[1]);
+                if (vc) y[o + jc] = __float2bfloat16_rn(b0[i][3] + c[3]);
+              }
+            }
           }
         }
       }
+      u += tile1 - tile0;
+      rem = 0;
+      ++job;
     }
   }
 }
@@ -276,19 +304,20 @@ cudaError_t launch_lora_shrink_stream(const PlanView& pv, ShrinkJobs jobs, int n
 
 cudaError_t launch_lora_expand_stream(const PlanView& pv, ExpandJobs jobs, float scale, int n_sms,
                                       cudaStream_t stream) {
-  long items = 0;
-  int rmax = 0;
+  int tps = 0, rmax = 0;
   for (int j = 0; j < jobs.n; ++j) {
-    jobs.rows_per_item[j] = jobs.d_out[j] <= 512 ? 128 : 512;
-    jobs.per_seg[j] = (jobs.d_out[j] + jobs.rows_per_item[j] - 1) / jobs.rows_per_item[j];
-    items += (long)pv.Smax * jobs.per_seg[j];
+    jobs.rows_per_item[j] = 16;
+    jobs.per_seg[j] = (jobs.d_out[j] + 15) / 16;   // 16-row tiles per segment
+    tps += jobs.per_seg[j];
     rmax = jobs.r[j] > rmax ? jobs.r[j] : rmax;
   }
-  const int grid = stream_grid(items, n_sms, 16);
+  // one warp per 2 tiles at least; at most one CTA per resident slot (4 per SM)
+  const long max_ctas = ((long)pv.Smax * tps + 2 * (kExpandThreads / 32) - 1) / (2 * (kExpandThreads / 32));
+  const int grid = stream_grid(max_ctas, n_sms, 4);
   if (rmax <= 32)
-    lora_expand_stream_kernel<1><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale);
+    lora_expand_stream_kernel<1><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale, tps);
   else
-    lora_expand_stream_kernel<2><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale);
+    lora_expand_stream_kernel<2><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale, tps);
   return cudaGetLastError();
 }
 
