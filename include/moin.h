@@ -93,7 +93,7 @@ typedef struct {
 enum {
   MOIN_K_ROUTE_SIMPLE = 0, MOIN_K_ROUTE_TC = 1, MOIN_K_ROUTE_FINISH = 2, MOIN_K_PLAN = 3, MOIN_K_GEMM_WARP = 4,
   MOIN_K_GEMM_TC = 5, MOIN_K_SHRINK_STREAM = 6, MOIN_K_EXPAND_STREAM = 7, MOIN_K_SHRINK_TC = 8,
-  MOIN_K_FUSED_TC = 9, MOIN_K_GLUE = 10, MOIN_K_ATTENTION = 11, MOIN_K_COUNT = 12
+  MOIN_K_FUSED_TC = 9, MOIN_K_GLUE = 10, MOIN_K_ATTENTION = 11, MOIN_K_ROUTE_CLUSTER = 12, MOIN_K_COUNT = 13
 };
 moin_status moin_profile_enable(int32_t capacity);
 moin_status moin_profile_read(moin_profile_record* out, int32_t capacity, int32_t* n);

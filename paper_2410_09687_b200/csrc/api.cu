@@ -164,7 +164,7 @@ moin_status moin_profile_read(moin_profile_record* out, int32_t capacity, int32_
 const char* moin_kernel_name(int32_t k) {
   static const char* names[MOIN_K_COUNT] = {"route_simple", "route_tc", "route_finish", "plan", "gemm_warp", "gemm_tc",
                                             "lora_shrink_stream", "lora_expand_stream", "lora_shrink_tc",
-                                            "lora_fused_tc", "decoder_glue", "attention"};
+                                            "lora_fused_tc", "decoder_glue", "attention", "route_cluster"};
   return (k >= 0 && k < MOIN_K_COUNT) ? names[k] : "unknown";
 }
 
@@ -205,6 +205,12 @@ moin_status moin_route(const moin_router* router, const void* queries, int32_t Q
   if (hs->gemm_impl == 2) {
     if (!tc_ok) return MOIN_ERR_BAD_SHAPE;
     use_tc = true;
+  }
+  if (hs->gemm_impl == 0 && route_cluster_supported(Q, K, D)) {   // decode-sized batch: one launch, no scratch
+    ProfScope prof(MOIN_K_ROUTE_CLUSTER, 1, s);
+    return record_cuda(launch_route_cluster((const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids,
+                                            router->inv_norm, router->centroid_to_expert, Q, K, D, out_expert,
+                                            out_centroid, out_best_sim, s));
   }
   if (use_tc) {
     if (!workspace || workspace_bytes < moin_route_workspace_bytes(Q, K, D) || !aligned16(workspace))
@@ -295,7 +301,7 @@ moin_status moin_plan_build(const int32_t* token_expert, moin_plan* plan, moin_s
   cudaStream_t s = (cudaStream_t)stream;
   PlanView v = plan_view(plan->buffer, plan->T, plan->E);
   {
-    ProfScope prof(MOIN_K_PLAN, plan->T > kPlanChunk ? 4 : 3, s);
+    ProfScope prof(MOIN_K_PLAN, plan_launches(plan->T, plan->E), s);
     st = record_cuda(launch_plan_build(token_expert, v, hs->status, s));
   }
   if (st) return st;

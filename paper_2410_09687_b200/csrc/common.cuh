@@ -108,6 +108,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 // Launchers implemented in the .cu files (host side).
+int plan_launches(int T, int E);   // kernels launch_plan_build issues for this shape
 cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, DeviceStatus* status, cudaStream_t stream);
 // Register-fed short-segment kernels: one launch covers up to kMaxStreamJobs projections sharing a plan.
 constexpr int kMaxStreamJobs = 4;
@@ -137,6 +138,10 @@ cudaError_t launch_inv_norm(const __nv_bfloat16* c, int K, int D, float* inv_nor
 cudaError_t launch_route_simple(const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
                                 const int* cmap, int Q, int K, int D, int* out_expert, int* out_centroid,
                                 float* out_best, cudaStream_t stream);
+bool route_cluster_supported(int Q, int K, int D);
+cudaError_t launch_route_cluster(const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
+                                 const int* cmap, int Q, int K, int D, int* out_expert, int* out_centroid,
+                                 float* out_best, cudaStream_t stream);
 cudaError_t launch_route_finish(const unsigned long long* keys, const __nv_bfloat16* q, const int* cmap, int Q, int D,
                                 int* out_expert, int* out_centroid, float* out_best, cudaStream_t stream);
 

@@ -1,6 +1,7 @@
 // Batch plan: grouping of tokens by expert id (integer work only).
 //
-// A few small launches:
+// Batches of up to 1024 tokens take one single-CTA launch (plan_small_kernel: a bitonic sort of
+// (expert id, token) keys in shared memory).  Larger ones take a few small launches:
 //   plan_rank_kernel    per 256-token chunk: sanitise ids, stable in-chunk rank, per-chunk histogram
 //   plan_prefix_kernel  (batches of more than one chunk) per expert id: prefix of its counts over the chunks
 //   plan_scan_kernel    one CTA: prefix over expert ids -> segment list; run tiles
@@ -113,6 +114,39 @@ __global__ void __launch_bounds__(256) plan_prefix_kernel(PlanView v) {
   v.keybase[k] = run;
 }
 
+// Row tiles: maximal runs of equal expert id in token order, cut every kTileRows rows.  One CTA of 1024
+// threads; `key[t]` is the sanitised id of token t (shared or global memory).  smem: 33 ints, s_carry: 2.
+__device__ __forceinline__ void plan_tiles(const PlanView& v, const int* key, int* smem, int* s_carry) {
+  const int tid = threadIdx.x;
+  const int T = v.T, E = v.E;
+  int carry_start = 0, carry_tiles = 0;
+  for (int t0 = 0; t0 < T; t0 += 1024) {
+    int t = t0 + tid;
+    int k = (t < T) ? key[t] : -3;
+    int is_start = (t < T) && (t == 0 || key[t - 1] != k);
+    int rs = block_incl_max_1024(is_start ? t : -1, smem);
+    rs = max(rs, carry_start);
+    int flag = (t < T) && (((t - rs) % kTileRows) == 0);
+    int tot;
+    int idx = carry_tiles + block_excl_sum_1024(flag, smem, &tot);
+    if (flag) {
+      v.tile_row0[idx] = t;
+      v.tile_expert[idx] = (k == E) ? -1 : k;
+    }
+    if (tid == 1023) s_carry[0] = rs;
+    __syncthreads();
+    carry_start = s_carry[0];
+    carry_tiles += tot;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    v.tile_row0[carry_tiles] = T;
+    v.header[PH_NTILES] = carry_tiles;
+  }
+  __syncthreads();
+  for (int i = tid; i < carry_tiles; i += 1024) v.tile_rows[i] = v.tile_row0[i + 1] - v.tile_row0[i];
+}
+
 __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_prefix) {
   __shared__ int smem[33];
   __shared__ int s_carry[2];
@@ -164,33 +198,84 @@ __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_pref
     v.header[PH_E] = E;
   }
 
-  // 3. row tiles: maximal runs of equal expert id in token order, cut every kTileRows rows
-  int carry_start = 0, carry_tiles = 0;
-  for (int t0 = 0; t0 < T; t0 += 1024) {
-    int t = t0 + tid;
-    int k = (t < T) ? v.key[t] : -3;
-    int is_start = (t < T) && (t == 0 || v.key[t - 1] != k);
-    int rs = block_incl_max_1024(is_start ? t : -1, smem);
-    rs = max(rs, carry_start);
-    int flag = (t < T) && (((t - rs) % kTileRows) == 0);
-    int tot;
-    int idx = carry_tiles + block_excl_sum_1024(flag, smem, &tot);
-    if (flag) {
-      v.tile_row0[idx] = t;
-      v.tile_expert[idx] = (k == E) ? -1 : k;
+  // 3. row tiles
+  plan_tiles(v, v.key, smem, s_carry);
+}
+
+// Whole plan of a batch of at most 1024 tokens in one CTA.  The tokens are sorted by the key
+// (sanitised expert id << 10 | token index) with a bitonic network in shared memory: the low bits make
+// the order stable, the sorted position of a token is its place in `perm`, and the segments are the
+// runs of equal id in the sorted sequence (ascending id, the "no adapter" bucket E last).
+constexpr int kPlanSmallT = 1024;
+constexpr int kPlanSmallE = 1 << 20;   // the id must fit above the 10 token bits of a 31-bit key
+__global__ void __launch_bounds__(1024) plan_small_kernel(const int* __restrict__ token_expert, PlanView v,
+                                                          DeviceStatus* status) {
+  __shared__ int s_key[kPlanSmallT];    // sanitised id by token
+  __shared__ int s_sort[kPlanSmallT];   // sort keys
+  __shared__ int smem[33];
+  __shared__ int s_carry[2];
+  const int tid = threadIdx.x;
+  const int T = v.T, E = v.E;
+  int k = 0x1FFFFF;  // padding sorts last
+  if (tid < T) {
+    int e = token_expert[tid];
+    if (e >= 0 && e < E) {
+      k = e;
+    } else {
+      k = E;  // "no adapter" bucket
+      if (e != -1) atomicAdd(&status->invalid_expert_ids, 1);
     }
-    if (tid == 1023) s_carry[0] = rs;
-    __syncthreads();
-    carry_start = s_carry[0];
-    carry_tiles += tot;
-    __syncthreads();
   }
-  if (tid == 0) {
-    v.tile_row0[carry_tiles] = T;
-    v.header[PH_NTILES] = carry_tiles;
-  }
+  s_key[tid] = (tid < T) ? k : -2;
+  s_sort[tid] = (k << 10) | tid;
+  int n = 32;
+  while (n < T) n <<= 1;
   __syncthreads();
-  for (int i = tid; i < carry_tiles; i += 1024) v.tile_rows[i] = v.tile_row0[i + 1] - v.tile_row0[i];
+  for (int size = 2; size <= n; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      const int partner = tid ^ stride;
+      if (tid < n && partner > tid) {
+        const int a = s_sort[tid], b = s_sort[partner];
+        const bool up = (tid & size) == 0;
+        if ((a > b) == up) {
+          s_sort[tid] = b;
+          s_sort[partner] = a;
+        }
+      }
+      __syncthreads();
+    }
+  }
+  // sorted position p holds (id, token): perm, run starts, segment list
+  const int mine = (tid < T) ? s_sort[tid] : 0x7FFFFFFF;
+  const int id = mine >> 10;
+  if (tid < T) v.perm[tid] = mine & 1023;
+  const int prev_id = (tid > 0 && tid <= T) ? (s_sort[tid - 1] >> 10) : -1;
+  const int is_start = (tid < T) && id < E && (tid == 0 || prev_id != id);
+  int n_seg;
+  const int seg = block_excl_sum_1024(is_start, smem, &n_seg);
+  if (is_start) {
+    v.seg_expert[seg] = id;
+    v.seg_start[seg] = tid;
+  }
+  // tokens with an adapter: positions before the first "no adapter" key
+  int n_lora;
+  block_excl_sum_1024((tid < T) && id < E, smem, &n_lora);
+  if (tid == 0) v.seg_start[n_seg] = n_lora;
+  __syncthreads();
+  int len = 0;
+  if (is_start) {
+    len = v.seg_start[seg + 1] - tid;
+    v.seg_tab[seg] = make_int4(id, tid, len, 0);
+  }
+  const int max_seg = block_incl_max_1024(len, smem);
+  if (tid == 1023) {
+    v.header[PH_NSEG] = n_seg;
+    v.header[PH_NLORA] = n_lora;
+    v.header[PH_MAXSEG] = max_seg;
+    v.header[PH_T] = T;
+    v.header[PH_E] = E;
+  }
+  plan_tiles(v, s_key, smem, s_carry);
 }
 
 __global__ void __launch_bounds__(kPlanChunk) plan_scatter_kernel(PlanView v) {
@@ -201,7 +286,16 @@ __global__ void __launch_bounds__(kPlanChunk) plan_scatter_kernel(PlanView v) {
   v.perm[pos] = t;
 }
 
+int plan_launches(int T, int E) {
+  if (T <= kPlanSmallT && E < kPlanSmallE) return 1;
+  return T > kPlanChunk ? 4 : 3;
+}
+
 cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, DeviceStatus* status, cudaStream_t stream) {
+  if (v.T <= kPlanSmallT && v.E < kPlanSmallE) {
+    plan_small_kernel<<<1, 1024, 0, stream>>>(token_expert, v, status);
+    return cudaGetLastError();
+  }
   cudaError_t e = cudaMemsetAsync(v.hist, 0, sizeof(int) * (size_t)v.n_chunks * (size_t)(v.E + 1), stream);
   if (e != cudaSuccess) return e;
   plan_rank_kernel<<<v.n_chunks, kPlanChunk, 0, stream>>>(token_expert, v.T, v.E, v.key, v.rank, v.hist, status);

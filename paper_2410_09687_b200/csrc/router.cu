@@ -1,6 +1,10 @@
 // Query router kernels: centroid inverse norms, the CUDA-core cosine-argmax kernel used for
 // small problems and odd shapes, and the finishing pass shared with the tensor-core router.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace moin {
 
@@ -146,6 +150,156 @@ route_finish_kernel(const unsigned long long* __restrict__ keys, const __nv_bflo
     ss = warp_sum(ss);
     if (lane == 0) out_best[i] = (key == 0ull) ? -INFINITY : key_to_float((uint32_t)(key >> 32)) * rsqrtf(ss);
   }
+}
+
+// ----------------------------------------------------------------------------------------
+// Small-batch router (decode-sized Q): one launch, no scratch memory.
+//
+// A cluster of kRcCluster CTAs serves kRcQ queries.  The centroids are cut into 16-row tiles,
+// dealt round-robin to the cluster's warps; a warp holds its tile's rows as the A operand of
+// m16n8k16 (loaded straight from global memory, 16 bytes per lane: lane t of a row group takes
+// k-elements 8t..8t+7 of every 32, and the queries, staged once in shared memory, are read with the
+// same k assignment, so the contraction is unchanged) and the kRcQ queries as kRcQ/8 B operands.
+// Every CTA merges its warps' per-query winners in its own shared memory with a 64-bit max on the
+// (similarity, index) key; after a cluster barrier CTA 0 reads the other CTAs' keys through
+// distributed shared memory and writes the result.
+// ----------------------------------------------------------------------------------------
+constexpr int kRcCluster = 8, kRcWarps = 4, kRcQ = 32, kRcUnroll = 6;
+
+__device__ __forceinline__ unsigned long long route_key(float sim, int k) {
+  uint32_t u = __float_as_uint(sim);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)k);
+}
+
+__global__ void __cluster_dims__(kRcCluster, 1, 1) __launch_bounds__(kRcWarps * 32)
+route_cluster_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ c,
+                     const float* __restrict__ inv_norm, const int* __restrict__ cmap, int Q, int K, int D,
+                     int* __restrict__ out_expert, int* __restrict__ out_centroid, float* __restrict__ out_best) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ unsigned long long s_keys[kRcQ];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const int rank = (int)cluster.block_rank();
+  const int q0 = (blockIdx.x / kRcCluster) * kRcQ;
+  const int pitch = D * 2 + 16;  // bytes; the 16-byte skew keeps the 8 rows of a fragment on distinct banks
+  const int nch = D / 8;
+  for (int i = tid; i < kRcQ * nch; i += kRcWarps * 32) {
+    const int qi = i / nch, ch = i - qi * nch;
+    const uint4 v = (q0 + qi < Q) ? ldg_cached(q + (size_t)(q0 + qi) * D + ch * 8) : make_uint4(0, 0, 0, 0);
+    *reinterpret_cast<uint4*>(smem_raw + (size_t)qi * pitch + ch * 16) = v;
+  }
+  if (tid < kRcQ) s_keys[tid] = 0ull;
+  __syncthreads();
+
+  const int n_tiles = (K + 15) / 16, steps = D / 32;
+  for (int tile = rank * kRcWarps + warp; tile < n_tiles; tile += kRcCluster * kRcWarps) {
+    const int r0 = tile * 16 + g, r1 = r0 + 8;
+    // rows past K read row K-1 (in bounds) and are masked below
+    const __nv_bfloat16* a0p = c + (size_t)min(r0, K - 1) * D + t * 8;
+    const __nv_bfloat16* a1p = c + (size_t)min(r1, K - 1) * D + t * 8;
+    float acc[kRcQ / 8][4];
+#pragma unroll
+    for (int j = 0; j < kRcQ / 8; ++j)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[j][e] = 0.f;
+    for (int s0 = 0; s0 < steps; s0 += kRcUnroll) {
+      uint4 a0[kRcUnroll], a1[kRcUnroll];
+#pragma unroll
+      for (int u = 0; u < kRcUnroll; ++u) {
+        const bool on = s0 + u < steps;
+        a0[u] = on ? ldg_cached(a0p + (s0 + u) * 32) : make_uint4(0, 0, 0, 0);
+        a1[u] = on ? ldg_cached(a1p + (s0 + u) * 32) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int u = 0; u < kRcUnroll; ++u) {
+        if (s0 + u >= steps) break;
+#pragma unroll
+        for (int j = 0; j < kRcQ / 8; ++j) {
+          const uint4 b = *reinterpret_cast<const uint4*>(smem_raw + (size_t)(j * 8 + g) * pitch + (s0 + u) * 64 + t * 16);
+          mma_bf16_16816(acc[j], a0[u].x, a1[u].x, a0[u].y, a1[u].y, b.x, b.y);
+          mma_bf16_16816(acc[j], a0[u].z, a1[u].z, a0[u].w, a1[u].w, b.z, b.w);
+        }
+      }
+    }
+    // acc[j][0..1]: centroid r0, queries j*8 + 2t, 2t+1;  acc[j][2..3]: centroid r1
+    const float inv0 = (r0 < K) ? inv_norm[r0] : 0.f, inv1 = (r1 < K) ? inv_norm[r1] : 0.f;
+#pragma unroll
+    for (int j = 0; j < kRcQ / 8; ++j)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float s_lo = acc[j][e] * inv0, s_hi = acc[j][2 + e] * inv1;
+        unsigned long long key = 0ull;   // 0 = no candidate (zero-norm or padding row, NaN or -inf similarity)
+        if (inv0 > 0.f && s_lo > -INFINITY) key = route_key(s_lo, r0);
+        if (inv1 > 0.f && s_hi > -INFINITY) {
+          const unsigned long long k1 = route_key(s_hi, r1);
+          key = k1 > key ? k1 : key;
+        }
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+          const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+          key = other > key ? other : key;
+        }
+        if (g == 0 && key != 0ull) atomicMax(&s_keys[j * 8 + 2 * t + e], key);
+      }
+  }
+  cluster.sync();
+  if (rank == 0) {
+    // one warp per query: lanes 0..kRcCluster-1 fetch the CTAs' keys, all lanes share the norm
+    for (int qi = warp; qi < kRcQ; qi += kRcWarps) {
+      if (q0 + qi >= Q) break;
+      unsigned long long key = 0ull;
+      if (lane < kRcCluster) key = *cluster.map_shared_rank(&s_keys[qi], lane);
+#pragma unroll
+      for (int o = 1; o < kRcCluster; o <<= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+        key = other > key ? other : key;
+      }
+      key = __shfl_sync(0xffffffffu, key, 0);
+      const int id = (key == 0ull) ? 0 : (int)(0xFFFFFFFFu - (uint32_t)(key & 0xFFFFFFFFull));
+      if (lane == 0) {
+        if (out_centroid) out_centroid[q0 + qi] = id;
+        out_expert[q0 + qi] = cmap ? cmap[id] : id;
+      }
+      if (out_best) {
+        float ss = 0.f;
+        for (int ch = lane; ch < nch; ch += 32) {
+          const uint4 v = *reinterpret_cast<const uint4*>(smem_raw + (size_t)qi * pitch + ch * 16);
+          const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            ss = fmaf(bf16_lo(w[e]), bf16_lo(w[e]), ss);
+            ss = fmaf(bf16_hi(w[e]), bf16_hi(w[e]), ss);
+          }
+        }
+        ss = warp_sum(ss);
+        if (lane == 0)
+          out_best[q0 + qi] = (key == 0ull) ? -INFINITY : key_to_float((uint32_t)(key >> 32)) * rsqrtf(ss);
+      }
+    }
+  }
+  cluster.sync();  // the other CTAs' shared memory stays alive until CTA 0 has read it
+}
+
+bool route_cluster_supported(int Q, int K, int D) {
+  return Q >= 1 && K >= 1 && (D % 32) == 0 && (size_t)kRcQ * (D * 2 + 16) <= 200 * 1024 &&
+         (long long)Q * K <= (1ll << 19);
+}
+
+cudaError_t launch_route_cluster(const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
+                                 const int* cmap, int Q, int K, int D, int* out_expert, int* out_centroid,
+                                 float* out_best, cudaStream_t stream) {
+  const size_t smem = (size_t)kRcQ * (D * 2 + 16);
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaError_t e = cudaFuncSetAttribute(route_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = smem;
+  }
+  const int groups = (Q + kRcQ - 1) / kRcQ;
+  route_cluster_kernel<<<groups * kRcCluster, kRcWarps * 32, smem, stream>>>(q, c, inv_norm, cmap, Q, K, D, out_expert,
+                                                                            out_centroid, out_best);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_inv_norm(const __nv_bfloat16* c, int K, int D, float* inv_norm, cudaStream_t stream) {

@@ -69,6 +69,16 @@ def test_plan_ragged_and_edge_cases():
     assert _check(rng.integers(0, 500, size=256).astype(np.int32), 500).mode == moin.PLAN_SEGMENTS
 
 
+def test_plan_single_launch_and_chunked_paths_at_the_switch():
+    # up to 1024 tokens: one single-CTA launch (shared-memory sort); beyond: the chunked launches
+    rng = np.random.default_rng(7)
+    for T, E in [(1024, 5000), (1025, 5000), (1023, 37), (200, 9000), (600, 70000), (33, 2), (31, 500), (513, 8)]:
+        te = rng.integers(-1, E, size=T).astype(np.int32)
+        te[rng.integers(0, T, size=T // 4)] = rng.integers(0, min(E, 6))   # a few long segments too
+        _check(te, E)
+    _check(np.repeat(rng.integers(0, 3, size=4), 256).astype(np.int32), 3)   # runs longer than one tile
+
+
 def test_plan_is_deterministic():
     rng = np.random.default_rng(4)
     te = torch.from_numpy(rng.integers(0, 100, size=5000).astype(np.int32)).to(DEV)

@@ -41,7 +41,7 @@ def test_router_tiny(impl):
     np.testing.assert_allclose(best, ref["best"], atol=2e-3)
 
 
-@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("impl", [0, 1, 2])   # 0: cluster kernel at this size, 1: CUDA cores, 2: tcgen05
 def test_router_decode_shape_with_map(impl):
     case = mi.planted_router(K=500, Q=256, D=768, seed=1)
     cmap = np.arange(500, dtype=np.int32)[::-1].copy()
@@ -71,6 +71,20 @@ def test_router_stress_full_size_sampled():
     assert_router_matches(cid[rows], ref)
 
 
+@pytest.mark.parametrize("Q,K,D", [(1, 1, 32), (33, 70, 64), (100, 17, 96), (257, 500, 768), (5, 5000, 768),
+                                   (1024, 512, 256), (40, 1000, 1504)])
+def test_router_small_batch_shapes(Q, K, D):
+    # decode-sized batches take the single-launch cluster kernel: ragged query groups, ragged
+    # centroid tiles, fewer tiles than warps in the cluster, several tiles per warp
+    case = mi.planted_router(K=K, Q=Q, D=D, seed=11 + Q)
+    cmap = np.random.default_rng(Q).permutation(K).astype(np.int32)
+    eid, cid, best = _route(case, cmap)
+    ref = _oracle(case, cmap)
+    assert_router_matches(cid, ref)
+    assert np.array_equal(eid, cmap[cid])
+    np.testing.assert_allclose(best, ref["best"], atol=2e-3)
+
+
 def test_router_near_tie_stress():
     # noise added to the UNIT centroid: many small margins; mismatches only allowed below the margin.
     case = mi.planted_router(K=1000, Q=2048, D=768, seed=5, unit_centroid_noise=True)
@@ -80,7 +94,7 @@ def test_router_near_tie_stress():
     print(f"near-ties (<{TIE_MARGIN}): {n_near}, of which differ: {n_diff}")
 
 
-@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("impl", [0, 1, 2])
 def test_router_degenerate_inputs(impl):
     rng = np.random.default_rng(6)
     c = torch.from_numpy(rng.normal(size=(70, 64))).to(torch.bfloat16)

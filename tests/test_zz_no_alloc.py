@@ -47,7 +47,8 @@ def test_static_router_matches_workspace_router_twice_in_a_row():
     ref2, got2 = _both(r_small, small.queries)
     assert torch.equal(ref2[0], got2[0]) and torch.equal(ref2[1], got2[1])
     assert torch.equal(got2[1].cpu(), small.labels.cpu())
-    np.testing.assert_allclose(got2[2].cpu().numpy(), ref2[2].cpu().numpy(), rtol=0, atol=0)
+    # a batch this small goes through another kernel in the workspace call: other summation order
+    np.testing.assert_allclose(got2[2].cpu().numpy(), ref2[2].cpu().numpy(), rtol=0, atol=2e-6)
     assert moin.device_status()["timeout_flag"] == 0
 
 
