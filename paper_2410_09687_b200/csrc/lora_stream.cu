@@ -13,9 +13,9 @@
 
 namespace moin {
 
-constexpr int kShrinkThreads = 256;      // 8 warps split the reduction dimension
+constexpr int kShrinkThreads = 128;      // 4 warps split the reduction dimension
 constexpr int kShrinkWarps = kShrinkThreads / 32;
-constexpr int kShrinkUnroll = 8;         // 32-wide k steps in flight per warp
+constexpr int kShrinkUnroll = 4;         // 32-wide k steps in flight per warp
 constexpr int kExpandThreads = 128;      // 4 warps
 constexpr int kExpandTilesPerBatch = 2;  // 16-row tiles whose loads are in flight together, per warp
 
@@ -68,8 +68,12 @@ __device__ __forceinline__ SegMeta load_seg(const int4* __restrict__ seg_tab, co
 }
 
 // h[pos][rho] = sum_i A[slot][rho][i] * x[perm[pos]][i]      (fp32, pos = position in sorted order)
-// Work item = (job, segment, group of 16 adapter rows); the CTA's 8 warps interleave over k.
-__global__ void __launch_bounds__(kShrinkThreads, 2)
+// Work item = (job, segment, group of 16 adapter rows); the CTA's warps interleave over k.
+// Small CTAs (4 warps, 80 registers: six per SM, and room beside a base-GEMM CTA) and one CTA per item:
+// the hardware's block scheduler hands the items out as slots free up, so a launch ends evenly whatever
+// the base GEMMs on the side streams occupy, and a CTA's metadata hops (segment count, table entry,
+// slot) hide behind the streams of the other CTAs on its SM.
+__global__ void __launch_bounds__(kShrinkThreads, 6)
 lora_shrink_stream_kernel(const int* __restrict__ header, const int* __restrict__ perm,
                           const int4* __restrict__ seg_tab, const ShrinkJobs jobs) {
   __shared__ float red[kShrinkWarps][32][4];
@@ -297,7 +301,8 @@ cudaError_t launch_lora_shrink_stream(const PlanView& pv, ShrinkJobs jobs, int n
     jobs.per_seg[j] = (jobs.r[j] + 15) / 16;
     items += (long)pv.Smax * jobs.per_seg[j];
   }
-  lora_shrink_stream_kernel<<<stream_grid(items, n_sms, 8), kShrinkThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab,
+  // one CTA per item (capped; CTAs stride over the items beyond the cap)
+  lora_shrink_stream_kernel<<<stream_grid(items, n_sms, 1024), kShrinkThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab,
                                                                                        jobs);
   return cudaGetLastError();
 }
