@@ -156,7 +156,8 @@ route_finish_kernel(const unsigned long long* __restrict__ keys, const __nv_bflo
 // Small-batch router (decode-sized Q): one launch, no scratch memory.
 //
 // A cluster of kRcCluster CTAs serves kRcQ queries.  The centroids are cut into 16-row tiles,
-// dealt round-robin to the cluster's warps; a warp holds its tile's rows as the A operand of
+// dealt round-robin to the cluster's warps (two warps share a tile, half of the k range each);
+// a warp holds its tile's rows as the A operand of
 // m16n8k16 (loaded straight from global memory, 16 bytes per lane: lane t of a row group takes
 // k-elements 8t..8t+7 of every 32, and the queries, staged once in shared memory, are read with the
 // same k assignment, so the contraction is unchanged) and the kRcQ queries as kRcQ/8 B operands.
@@ -164,7 +165,8 @@ route_finish_kernel(const unsigned long long* __restrict__ keys, const __nv_bflo
 // (similarity, index) key; after a cluster barrier CTA 0 reads the other CTAs' keys through
 // distributed shared memory and writes the result.
 // ----------------------------------------------------------------------------------------
-constexpr int kRcCluster = 8, kRcWarps = 4, kRcQ = 32, kRcUnroll = 6;
+constexpr int kRcCluster = 8, kRcTileWarps = 4, kRcKSplit = 2, kRcWarps = kRcTileWarps * kRcKSplit, kRcQ = 32,
+              kRcUnroll = 12;
 
 __device__ __forceinline__ unsigned long long route_key(float sim, int k) {
   uint32_t u = __float_as_uint(sim);
@@ -172,48 +174,71 @@ __device__ __forceinline__ unsigned long long route_key(float sim, int k) {
   return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)k);
 }
 
+// Warp w works on centroid tile (w % kRcTileWarps) of the CTA's current round and on the
+// (w / kRcTileWarps)-th part of the k range; the parts are added in shared memory in a fixed order.
 __global__ void __cluster_dims__(kRcCluster, 1, 1) __launch_bounds__(kRcWarps * 32)
 route_cluster_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ c,
                      const float* __restrict__ inv_norm, const int* __restrict__ cmap, int Q, int K, int D,
                      int* __restrict__ out_expert, int* __restrict__ out_centroid, float* __restrict__ out_best) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ unsigned long long s_keys[kRcQ];
+  __shared__ float s_part[kRcTileWarps][kRcQ / 8][4][32];
   cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const int tw = warp % kRcTileWarps, kpart = warp / kRcTileWarps;
   const int rank = (int)cluster.block_rank();
   const int q0 = (blockIdx.x / kRcCluster) * kRcQ;
   const int pitch = D * 2 + 16;  // bytes; the 16-byte skew keeps the 8 rows of a fragment on distinct banks
   const int nch = D / 8;
-  for (int i = tid; i < kRcQ * nch; i += kRcWarps * 32) {
-    const int qi = i / nch, ch = i - qi * nch;
-    const uint4 v = (q0 + qi < Q) ? ldg_cached(q + (size_t)(q0 + qi) * D + ch * 8) : make_uint4(0, 0, 0, 0);
-    *reinterpret_cast<uint4*>(smem_raw + (size_t)qi * pitch + ch * 16) = v;
+  const int n_tiles = (K + 15) / 16, steps = D / 32;
+  const int steps_part = (steps + kRcKSplit - 1) / kRcKSplit;
+  const int s_lo = kpart * steps_part, s_hi = min(steps, s_lo + steps_part);
+
+  // the first batch of centroid rows is requested before the queries are staged: one round trip for both
+  int tile = rank * kRcTileWarps + tw;
+  uint4 a0[kRcUnroll], a1[kRcUnroll];
+  auto load_a = [&](int tl, int s0) {
+    const int r0 = tl * 16 + g, r1 = r0 + 8;
+    // rows past K read row K-1 (in bounds) and are masked at the end
+    const __nv_bfloat16* a0p = c + (size_t)min(r0, K - 1) * D + t * 8;
+    const __nv_bfloat16* a1p = c + (size_t)min(r1, K - 1) * D + t * 8;
+#pragma unroll
+    for (int u = 0; u < kRcUnroll; ++u) {
+      const bool on = tl < n_tiles && s0 + u < s_hi;
+      a0[u] = on ? ldg_cached(a0p + (s0 + u) * 32) : make_uint4(0, 0, 0, 0);
+      a1[u] = on ? ldg_cached(a1p + (s0 + u) * 32) : make_uint4(0, 0, 0, 0);
+    }
+  };
+  load_a(tile, s_lo);
+  for (int i0 = 0; i0 < kRcQ * nch; i0 += kRcWarps * 32 * 8) {
+    uint4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * kRcWarps * 32 + tid;
+      const int qi = i / nch, ch = i - qi * nch;
+      v[u] = (i < kRcQ * nch && q0 + qi < Q) ? ldg_cached(q + (size_t)(q0 + qi) * D + ch * 8) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * kRcWarps * 32 + tid;
+      const int qi = i / nch, ch = i - qi * nch;
+      if (i < kRcQ * nch) *reinterpret_cast<uint4*>(smem_raw + (size_t)qi * pitch + ch * 16) = v[u];
+    }
   }
   if (tid < kRcQ) s_keys[tid] = 0ull;
   __syncthreads();
 
-  const int n_tiles = (K + 15) / 16, steps = D / 32;
-  for (int tile = rank * kRcWarps + warp; tile < n_tiles; tile += kRcCluster * kRcWarps) {
-    const int r0 = tile * 16 + g, r1 = r0 + 8;
-    // rows past K read row K-1 (in bounds) and are masked below
-    const __nv_bfloat16* a0p = c + (size_t)min(r0, K - 1) * D + t * 8;
-    const __nv_bfloat16* a1p = c + (size_t)min(r1, K - 1) * D + t * 8;
+  for (bool first = true; tile - tw < n_tiles; tile += kRcCluster * kRcTileWarps, first = false) {   // CTA-uniform trip count
     float acc[kRcQ / 8][4];
 #pragma unroll
     for (int j = 0; j < kRcQ / 8; ++j)
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[j][e] = 0.f;
-    for (int s0 = 0; s0 < steps; s0 += kRcUnroll) {
-      uint4 a0[kRcUnroll], a1[kRcUnroll];
+    for (int s0 = s_lo; s0 < s_hi; s0 += kRcUnroll) {
+      if (!first || s0 > s_lo) load_a(tile, s0);
 #pragma unroll
       for (int u = 0; u < kRcUnroll; ++u) {
-        const bool on = s0 + u < steps;
-        a0[u] = on ? ldg_cached(a0p + (s0 + u) * 32) : make_uint4(0, 0, 0, 0);
-        a1[u] = on ? ldg_cached(a1p + (s0 + u) * 32) : make_uint4(0, 0, 0, 0);
-      }
-#pragma unroll
-      for (int u = 0; u < kRcUnroll; ++u) {
-        if (s0 + u >= steps) break;
+        if (s0 + u >= s_hi) break;
 #pragma unroll
         for (int j = 0; j < kRcQ / 8; ++j) {
           const uint4 b = *reinterpret_cast<const uint4*>(smem_raw + (size_t)(j * 8 + g) * pitch + (s0 + u) * 64 + t * 16);
@@ -222,26 +247,42 @@ route_cluster_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         }
       }
     }
-    // acc[j][0..1]: centroid r0, queries j*8 + 2t, 2t+1;  acc[j][2..3]: centroid r1
-    const float inv0 = (r0 < K) ? inv_norm[r0] : 0.f, inv1 = (r1 < K) ? inv_norm[r1] : 0.f;
+    // add the k parts: part 1.. hand their sums to part 0 through shared memory
+    if (kpart > 0) {
 #pragma unroll
-    for (int j = 0; j < kRcQ / 8; ++j)
+      for (int j = 0; j < kRcQ / 8; ++j)
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const float s_lo = acc[j][e] * inv0, s_hi = acc[j][2 + e] * inv1;
-        unsigned long long key = 0ull;   // 0 = no candidate (zero-norm or padding row, NaN or -inf similarity)
-        if (inv0 > 0.f && s_lo > -INFINITY) key = route_key(s_lo, r0);
-        if (inv1 > 0.f && s_hi > -INFINITY) {
-          const unsigned long long k1 = route_key(s_hi, r1);
-          key = k1 > key ? k1 : key;
+        for (int e = 0; e < 4; ++e) s_part[tw][j][e][lane] = acc[j][e];
+    }
+    __syncthreads();
+    if (kpart == 0 && tile < n_tiles) {
+#pragma unroll
+      for (int j = 0; j < kRcQ / 8; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[j][e] += s_part[tw][j][e][lane];
+      // acc[j][0..1]: centroid r0, queries j*8 + 2t, 2t+1;  acc[j][2..3]: centroid r1
+      const int r0 = tile * 16 + g, r1 = r0 + 8;
+      const float inv0 = (r0 < K) ? inv_norm[r0] : 0.f, inv1 = (r1 < K) ? inv_norm[r1] : 0.f;
+#pragma unroll
+      for (int j = 0; j < kRcQ / 8; ++j)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const float sim0 = acc[j][e] * inv0, sim1 = acc[j][2 + e] * inv1;
+          unsigned long long key = 0ull;   // 0 = no candidate (zero-norm or padding row, NaN or -inf similarity)
+          if (inv0 > 0.f && sim0 > -INFINITY) key = route_key(sim0, r0);
+          if (inv1 > 0.f && sim1 > -INFINITY) {
+            const unsigned long long k1 = route_key(sim1, r1);
+            key = k1 > key ? k1 : key;
+          }
+#pragma unroll
+          for (int o = 4; o < 32; o <<= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+            key = other > key ? other : key;
+          }
+          if (g == 0 && key != 0ull) atomicMax(&s_keys[j * 8 + 2 * t + e], key);
         }
-#pragma unroll
-        for (int o = 4; o < 32; o <<= 1) {
-          const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
-          key = other > key ? other : key;
-        }
-        if (g == 0 && key != 0ull) atomicMax(&s_keys[j * 8 + 2 * t + e], key);
-      }
+    }
+    __syncthreads();   // s_part is free again
   }
   cluster.sync();
   if (rank == 0) {
