@@ -42,8 +42,9 @@ __global__ void __launch_bounds__(kPlanChunk) plan_rank_kernel(const int* __rest
   if (after == 0) hist[(size_t)blockIdx.x * (size_t)(E + 1) + k] = before + 1;
 }
 
-// Block-wide scans for 1024 threads.  `smem` must hold 33 ints.
-__device__ __forceinline__ int block_excl_sum_1024(int v, int* smem, int* total) {
+// Block-wide scans for NT threads (a multiple of 32, at most 1024).  `smem` must hold 33 ints.
+template <int NT>
+__device__ __forceinline__ int block_excl_sum(int v, int* smem, int* total) {
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int inc = v;
 #pragma unroll
@@ -55,7 +56,7 @@ __device__ __forceinline__ int block_excl_sum_1024(int v, int* smem, int* total)
   if (lane == 31) smem[w] = inc;
   __syncthreads();
   if (w == 0) {
-    int s = smem[lane];
+    int s = (lane < NT / 32) ? smem[lane] : 0;
     int si = s;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -69,7 +70,8 @@ __device__ __forceinline__ int block_excl_sum_1024(int v, int* smem, int* total)
   *total = smem[32];
   return smem[w] + inc - v;
 }
-__device__ __forceinline__ int block_incl_max_1024(int v, int* smem) {
+template <int NT>
+__device__ __forceinline__ int block_incl_max(int v, int* smem) {
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int inc = v;
 #pragma unroll
@@ -81,7 +83,7 @@ __device__ __forceinline__ int block_incl_max_1024(int v, int* smem) {
   if (lane == 31) smem[w] = inc;
   __syncthreads();
   if (w == 0) {
-    int s = smem[lane];
+    int s = (lane < NT / 32) ? smem[lane] : INT_MIN;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       int n = __shfl_up_sync(0xffffffffu, s, o);
@@ -114,26 +116,30 @@ __global__ void __launch_bounds__(256) plan_prefix_kernel(PlanView v) {
   v.keybase[k] = run;
 }
 
-// Row tiles: maximal runs of equal expert id in token order, cut every kTileRows rows.  One CTA of 1024
+// Row tiles: maximal runs of equal expert id in token order, cut every kTileRows rows.  One CTA of NT
 // threads; `key[t]` is the sanitised id of token t (shared or global memory).  smem: 33 ints, s_carry: 2.
-__device__ __forceinline__ void plan_tiles(const PlanView& v, const int* key, int* smem, int* s_carry) {
+// `row0` is where the tile starts are read back from to form the tile lengths: v.tile_row0 itself, or a
+// shared-memory copy ([T + 1] ints) when the caller has one.
+template <int NT>
+__device__ __forceinline__ void plan_tiles(const PlanView& v, const int* key, int* smem, int* s_carry, int* row0) {
   const int tid = threadIdx.x;
   const int T = v.T, E = v.E;
   int carry_start = 0, carry_tiles = 0;
-  for (int t0 = 0; t0 < T; t0 += 1024) {
+  for (int t0 = 0; t0 < T; t0 += NT) {
     int t = t0 + tid;
     int k = (t < T) ? key[t] : -3;
     int is_start = (t < T) && (t == 0 || key[t - 1] != k);
-    int rs = block_incl_max_1024(is_start ? t : -1, smem);
+    int rs = block_incl_max<NT>(is_start ? t : -1, smem);
     rs = max(rs, carry_start);
     int flag = (t < T) && (((t - rs) % kTileRows) == 0);
     int tot;
-    int idx = carry_tiles + block_excl_sum_1024(flag, smem, &tot);
+    int idx = carry_tiles + block_excl_sum<NT>(flag, smem, &tot);
     if (flag) {
       v.tile_row0[idx] = t;
+      if (row0 != v.tile_row0) row0[idx] = t;
       v.tile_expert[idx] = (k == E) ? -1 : k;
     }
-    if (tid == 1023) s_carry[0] = rs;
+    if (tid == NT - 1) s_carry[0] = rs;
     __syncthreads();
     carry_start = s_carry[0];
     carry_tiles += tot;
@@ -141,13 +147,15 @@ __device__ __forceinline__ void plan_tiles(const PlanView& v, const int* key, in
   }
   if (tid == 0) {
     v.tile_row0[carry_tiles] = T;
+    if (row0 != v.tile_row0) row0[carry_tiles] = T;
     v.header[PH_NTILES] = carry_tiles;
   }
   __syncthreads();
-  for (int i = tid; i < carry_tiles; i += 1024) v.tile_rows[i] = v.tile_row0[i + 1] - v.tile_row0[i];
+  for (int i = tid; i < carry_tiles; i += NT) v.tile_rows[i] = row0[i + 1] - row0[i];
 }
 
 __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_prefix) {
+  constexpr int NT = 1024;
   __shared__ int smem[33];
   __shared__ int s_carry[2];
   const int tid = threadIdx.x;
@@ -173,8 +181,8 @@ __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_pref
     int k = k0 + tid;
     int n = (k < E) ? v.keybase[k] : 0;
     int tot_tok, tot_seg;
-    int ex_tok = block_excl_sum_1024(n, smem, &tot_tok);
-    int ex_seg = block_excl_sum_1024(n > 0 ? 1 : 0, smem, &tot_seg);
+    int ex_tok = block_excl_sum<NT>(n, smem, &tot_tok);
+    int ex_seg = block_excl_sum<NT>(n > 0 ? 1 : 0, smem, &tot_seg);
     if (k < E) {
       v.keybase[k] = carry_tok + ex_tok;
       if (n > 0) {
@@ -187,7 +195,7 @@ __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_pref
     carry_tok += tot_tok;
     carry_seg += tot_seg;
   }
-  max_seg = block_incl_max_1024(max_seg, smem);
+  max_seg = block_incl_max<NT>(max_seg, smem);
   if (tid == 1023) {
     v.seg_start[carry_seg] = carry_tok;
     v.keybase[E] = carry_tok;
@@ -199,7 +207,7 @@ __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_pref
   }
 
   // 3. row tiles
-  plan_tiles(v, v.key, smem, s_carry);
+  plan_tiles<NT>(v, v.key, smem, s_carry, v.tile_row0);
 }
 
 // Whole plan of a batch of at most 1024 tokens in one CTA.  The tokens are sorted by the key
@@ -208,10 +216,12 @@ __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_pref
 // runs of equal id in the sorted sequence (ascending id, the "no adapter" bucket E last).
 constexpr int kPlanSmallT = 1024;
 constexpr int kPlanSmallE = 1 << 20;   // the id must fit above the 10 token bits of a 31-bit key
-__global__ void __launch_bounds__(1024) plan_small_kernel(const int* __restrict__ token_expert, PlanView v,
-                                                          DeviceStatus* status) {
-  __shared__ int s_key[kPlanSmallT];    // sanitised id by token
-  __shared__ int s_sort[kPlanSmallT];   // sort keys
+template <int NT>   // threads = sort width: the power of two at or above T, at least 128
+__global__ void __launch_bounds__(NT) plan_small_kernel(const int* __restrict__ token_expert, PlanView v,
+                                                        DeviceStatus* status) {
+  __shared__ int s_key[NT];        // sanitised id by token
+  __shared__ int s_sort[NT];       // sort keys, then the segment starts
+  __shared__ int s_row0[NT + 1];   // tile starts
   __shared__ int smem[33];
   __shared__ int s_carry[2];
   const int tid = threadIdx.x;
@@ -228,13 +238,11 @@ __global__ void __launch_bounds__(1024) plan_small_kernel(const int* __restrict_
   }
   s_key[tid] = (tid < T) ? k : -2;
   s_sort[tid] = (k << 10) | tid;
-  int n = 32;
-  while (n < T) n <<= 1;
   __syncthreads();
-  for (int size = 2; size <= n; size <<= 1) {
+  for (int size = 2; size <= NT; size <<= 1) {
     for (int stride = size >> 1; stride > 0; stride >>= 1) {
       const int partner = tid ^ stride;
-      if (tid < n && partner > tid) {
+      if (partner > tid) {
         const int a = s_sort[tid], b = s_sort[partner];
         const bool up = (tid & size) == 0;
         if ((a > b) == up) {
@@ -246,36 +254,35 @@ __global__ void __launch_bounds__(1024) plan_small_kernel(const int* __restrict_
     }
   }
   // sorted position p holds (id, token): perm, run starts, segment list
-  const int mine = (tid < T) ? s_sort[tid] : 0x7FFFFFFF;
+  const int mine = s_sort[tid];
   const int id = mine >> 10;
   if (tid < T) v.perm[tid] = mine & 1023;
-  const int prev_id = (tid > 0 && tid <= T) ? (s_sort[tid - 1] >> 10) : -1;
+  const int prev_id = (tid > 0) ? (s_sort[tid - 1] >> 10) : -1;
   const int is_start = (tid < T) && id < E && (tid == 0 || prev_id != id);
-  int n_seg;
-  const int seg = block_excl_sum_1024(is_start, smem, &n_seg);
-  if (is_start) {
-    v.seg_expert[seg] = id;
-    v.seg_start[seg] = tid;
-  }
-  // tokens with an adapter: positions before the first "no adapter" key
-  int n_lora;
-  block_excl_sum_1024((tid < T) && id < E, smem, &n_lora);
-  if (tid == 0) v.seg_start[n_seg] = n_lora;
+  int n_seg, n_lora;
+  const int seg = block_excl_sum<NT>(is_start, smem, &n_seg);
+  block_excl_sum<NT>((tid < T) && id < E, smem, &n_lora);   // tokens with an adapter sort first
+  __syncthreads();                                           // every thread has read its neighbour's key
+  if (is_start) s_sort[seg] = tid;                           // reuse as the segment-start list
+  if (tid == 0) s_sort[n_seg] = n_lora;
   __syncthreads();
   int len = 0;
   if (is_start) {
-    len = v.seg_start[seg + 1] - tid;
+    len = s_sort[seg + 1] - tid;
+    v.seg_expert[seg] = id;
+    v.seg_start[seg] = tid;
     v.seg_tab[seg] = make_int4(id, tid, len, 0);
   }
-  const int max_seg = block_incl_max_1024(len, smem);
-  if (tid == 1023) {
+  if (tid == 0) v.seg_start[n_seg] = n_lora;
+  const int max_seg = block_incl_max<NT>(len, smem);
+  if (tid == NT - 1) {
     v.header[PH_NSEG] = n_seg;
     v.header[PH_NLORA] = n_lora;
     v.header[PH_MAXSEG] = max_seg;
     v.header[PH_T] = T;
     v.header[PH_E] = E;
   }
-  plan_tiles(v, s_key, smem, s_carry);
+  plan_tiles<NT>(v, s_key, smem, s_carry, s_row0);
 }
 
 __global__ void __launch_bounds__(kPlanChunk) plan_scatter_kernel(PlanView v) {
@@ -293,7 +300,10 @@ int plan_launches(int T, int E) {
 
 cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, DeviceStatus* status, cudaStream_t stream) {
   if (v.T <= kPlanSmallT && v.E < kPlanSmallE) {
-    plan_small_kernel<<<1, 1024, 0, stream>>>(token_expert, v, status);
+    if (v.T <= 128) plan_small_kernel<128><<<1, 128, 0, stream>>>(token_expert, v, status);
+    else if (v.T <= 256) plan_small_kernel<256><<<1, 256, 0, stream>>>(token_expert, v, status);
+    else if (v.T <= 512) plan_small_kernel<512><<<1, 512, 0, stream>>>(token_expert, v, status);
+    else plan_small_kernel<1024><<<1, 1024, 0, stream>>>(token_expert, v, status);
     return cudaGetLastError();
   }
   cudaError_t e = cudaMemsetAsync(v.hist, 0, sizeof(int) * (size_t)v.n_chunks * (size_t)(v.E + 1), stream);
