@@ -323,8 +323,9 @@ route_cluster_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
 }
 
 bool route_cluster_supported(int Q, int K, int D) {
-  return Q >= 1 && K >= 1 && (D % 32) == 0 && (size_t)kRcQ * (D * 2 + 16) <= 200 * 1024 &&
-         (long long)Q * K <= (1ll << 19);
+  // few queries and at most two rounds of centroid tiles per cluster: beyond that the tensor-core GEMM wins
+  return Q >= 1 && Q <= 1024 && K >= 1 && K <= 16 * 2 * kRcCluster * kRcTileWarps && (D % 32) == 0 &&
+         (size_t)kRcQ * (D * 2 + 16) <= 200 * 1024;
 }
 
 cudaError_t launch_route_cluster(const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,

@@ -74,8 +74,9 @@ def test_router_stress_full_size_sampled():
 @pytest.mark.parametrize("Q,K,D", [(1, 1, 32), (33, 70, 64), (100, 17, 96), (257, 500, 768), (5, 5000, 768),
                                    (1024, 512, 256), (40, 1000, 1504)])
 def test_router_small_batch_shapes(Q, K, D):
-    # decode-sized batches take the single-launch cluster kernel: ragged query groups, ragged
-    # centroid tiles, fewer tiles than warps in the cluster, several tiles per warp
+    # decode-sized batches (up to 1024 queries and 1024 centroids) take the single-launch cluster kernel:
+    # ragged query groups, ragged centroid tiles, fewer tiles than warps in the cluster, two tiles per
+    # warp; (5, 5000) is past the switch and takes the tensor-core GEMM
     case = mi.planted_router(K=K, Q=Q, D=D, seed=11 + Q)
     cmap = np.random.default_rng(Q).permutation(K).astype(np.int32)
     eid, cid, best = _route(case, cmap)
