@@ -117,15 +117,30 @@ swiglu_kernel(__nv_bfloat16* __restrict__ gate, const __nv_bfloat16* __restrict_
 }
 
 // Causal grouped-query attention inside each request, head_dim 64.
-// Grid (query block of 64 rows, head, request); 4 warps x 16 query rows; keys/values staged
-// 64 at a time in shared memory (K as [key][dim], V transposed as [dim][key]); online softmax.
-constexpr int kAttPitch = 72;
+// Grid (query block of 64 rows, head, request); 4 warps x 16 query rows; keys and values staged 64 at a
+// time, row-major [key][dim], in a two-buffer shared-memory ring filled with 16-byte asynchronous copies
+// (the next tile is on its way while the current one is used); K fragments come from ldmatrix, V
+// fragments from ldmatrix.trans (the transpose P V needs); online softmax in the exp2 domain.
+constexpr int kAttPitch = 72;   // elements: 144-byte rows keep the 8 rows of an ldmatrix tile on distinct banks
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, bool valid) {
+  const int n = valid ? 16 : 0;   // 0 source bytes: the 16 destination bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_plain(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+
 __global__ void __launch_bounds__(128)
 attention_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                  const __nv_bfloat16* __restrict__ v, const int* __restrict__ cu, __nv_bfloat16* __restrict__ out,
                  int n_heads, int n_kv_heads, float scale_log2) {
-  __shared__ __align__(16) uint16_t Ks[64 * kAttPitch];
-  __shared__ __align__(16) uint16_t Vt[64 * kAttPitch];
+  __shared__ __align__(16) uint16_t Ks[2][64 * kAttPitch];
+  __shared__ __align__(16) uint16_t Vs[2][64 * kAttPitch];
   const int req = blockIdx.z, head = blockIdx.y, qb = blockIdx.x;
   const int t0 = cu[req], L = cu[req + 1] - t0;
   if (qb * 64 >= L) return;
@@ -133,6 +148,25 @@ attention_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
   const int qd = n_heads * 64, kvd = n_kv_heads * 64;
   const int r0 = qb * 64 + warp * 16 + g, r1 = r0 + 8;  // query rows (within request) of this thread
+  const int kv_end = min(L, qb * 64 + 64);
+  const uint32_t ks_base = (uint32_t)__cvta_generic_to_shared(&Ks[0][0]);
+  const uint32_t vs_base = (uint32_t)__cvta_generic_to_shared(&Vs[0][0]);
+  constexpr uint32_t kBufBytes = 64 * kAttPitch * 2;
+
+  auto stage = [&](int kb, int buf) {   // keys kb .. kb+63 -> buffer `buf`; rows past the request are zero-filled
+#pragma unroll
+    for (int i = tid; i < 64 * 8; i += 128) {
+      const int key = i >> 3, ch = i & 7;
+      const bool ok = kb + key < L;
+      const size_t row = (size_t)(t0 + (ok ? kb + key : L - 1)) * kvd + kvh * 64 + ch * 8;
+      const uint32_t off = (uint32_t)buf * kBufBytes + (uint32_t)(key * kAttPitch + ch * 8) * 2;
+      cp_async_16(ks_base + off, k + row, ok);
+      cp_async_16(vs_base + off, v + row, ok);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  stage(0, 0);
+
   uint32_t qa[4][4];
 #pragma unroll
   for (int ks = 0; ks < 4; ++ks) {
@@ -150,35 +184,31 @@ attention_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
 #pragma unroll
     for (int j = 0; j < 4; ++j) o[i][j] = 0.f;
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-  const int kv_end = min(L, qb * 64 + 64);
-  for (int kb = 0; kb < kv_end; kb += 64) {
-    __syncthreads();
-    for (int i = tid; i < 64 * 8; i += 128) {
-      const int key = i >> 3, ch = i & 7;
-      uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
-      if (kb + key < L) {
-        kv4 = ldg_cached(k + (size_t)(t0 + kb + key) * kvd + kvh * 64 + ch * 8);
-        vv4 = ldg_cached(v + (size_t)(t0 + kb + key) * kvd + kvh * 64 + ch * 8);
-      }
-      *reinterpret_cast<uint4*>(&Ks[key * kAttPitch + ch * 8]) = kv4;
-      const uint32_t w[4] = {vv4.x, vv4.y, vv4.z, vv4.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        Vt[(ch * 8 + 2 * e) * kAttPitch + key] = (uint16_t)(w[e] & 0xFFFFu);
-        Vt[(ch * 8 + 2 * e + 1) * kAttPitch + key] = (uint16_t)(w[e] >> 16);
-      }
+  // ldmatrix lane roles: lane l addresses row (l & 7) of matrix (l >> 3)
+  const int lm_row = lane & 7, lm_mat = lane >> 3;
+  for (int kb = 0, it = 0; kb < kv_end; kb += 64, ++it) {
+    const int buf = it & 1;
+    __syncthreads();                       // the other buffer's readers (previous tile) are done
+    if (kb + 64 < kv_end) {
+      stage(kb + 64, buf ^ 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
-    __syncthreads();
+    __syncthreads();                       // every thread's copies of this tile have landed
+    const uint32_t kbuf = ks_base + (uint32_t)buf * kBufBytes, vbuf = vs_base + (uint32_t)buf * kBufBytes;
     float s[8][4];
 #pragma unroll
     for (int nt = 0; nt < 8; ++nt) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) s[nt][j] = 0.f;
 #pragma unroll
-      for (int ks = 0; ks < 4; ++ks) {
-        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(&Ks[(nt * 8 + g) * kAttPitch + ks * 16 + 2 * t]);
-        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(&Ks[(nt * 8 + g) * kAttPitch + ks * 16 + 2 * t + 8]);
-        mma_bf16_16816(s[nt], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+      for (int kp = 0; kp < 2; ++kp) {
+        // matrices: keys nt*8.., dim chunks kp*32 + {0, 8, 16, 24}  ->  (b0, b1) of k-step 2kp and of 2kp+1
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4_plain(kbuf + (uint32_t)((nt * 8 + lm_row) * kAttPitch + kp * 32 + lm_mat * 8) * 2, b0, b1, b2, b3);
+        mma_bf16_16816(s[nt], qa[2 * kp][0], qa[2 * kp][1], qa[2 * kp][2], qa[2 * kp][3], b0, b1);
+        mma_bf16_16816(s[nt], qa[2 * kp + 1][0], qa[2 * kp + 1][1], qa[2 * kp + 1][2], qa[2 * kp + 1][3], b2, b3);
       }
     }
     // scale, causal mask, running max
@@ -217,12 +247,15 @@ attention_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
       pa[ks][hi * 2 + 1] = pack_bf16(p2, p3);
     }
 #pragma unroll
-    for (int dt = 0; dt < 8; ++dt)
+    for (int dp = 0; dp < 4; ++dp)
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks) {
-        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(&Vt[(dt * 8 + g) * kAttPitch + ks * 16 + 2 * t]);
-        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(&Vt[(dt * 8 + g) * kAttPitch + ks * 16 + 2 * t + 8]);
-        mma_bf16_16816(o[dt], pa[ks][0], pa[ks][1], pa[ks][2], pa[ks][3], b0, b1);
+        // matrices: keys ks*16 + {0, 8} x dims (2dp)*8.., then the same keys x dims (2dp+1)*8..; transposed on load
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4_trans(vbuf + (uint32_t)((ks * 16 + (lm_mat & 1) * 8 + lm_row) * kAttPitch + (2 * dp + (lm_mat >> 1)) * 8) * 2,
+                          b0, b1, b2, b3);
+        mma_bf16_16816(o[2 * dp], pa[ks][0], pa[ks][1], pa[ks][2], pa[ks][3], b0, b1);
+        mma_bf16_16816(o[2 * dp + 1], pa[ks][0], pa[ks][1], pa[ks][2], pa[ks][3], b2, b3);
       }
   }
   l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
