@@ -40,6 +40,8 @@ struct TcParams {
   const int* slot_of_expert;
   int tail_r;                  // EPI_STORE with plan: LoRA rank of the appended K block (0 = none)
   int rows_per_slot;           // rows of the B-side pool tensor per adapter slot (d_out, or r for EPI_SHRINK)
+  int b_box_rows;              // rows of the B-side TMA box when it is shorter than the tile's BN (0 = BN); the
+                               // rest of the stage's B region keeps stale bytes, whose columns nobody stores
   __nv_bfloat16* y;            // EPI_STORE / EPI_SHRINK output, leading dimension ldy
   __nv_bfloat16* y_lo;         // EPI_SHRINK: low part, value - bf16(value), same layout as y
   float* y0;                   // EPI_STORE: optional fp32 copy
@@ -153,7 +155,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t s = it % S, ph = (it / S) & 1u;
           if (!(ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag, p.status, 1))) break;
           const uint32_t sa = tiles_base + s * Cfg::kStageBytes, sb = sa + kBM * kBK * 2;
-          mbar_expect_tx(full0 + 8 * s, Cfg::kStageBytes);
+          const uint32_t b_rows = (kb < nkb_main && p.b_box_rows > 0) ? (uint32_t)p.b_box_rows : (uint32_t)BN;
+          mbar_expect_tx(full0 + 8 * s, (kBM + b_rows) * kBK * 2);
           if (kb < nkb_main) {
             tma_load_2d(sa, &tmA, full0 + 8 * s, kb * kBK, row0);
             tma_load_2d(sb, &tmB, full0 + 8 * s, kb * kBK, brow);
@@ -400,7 +403,7 @@ moin_status launch_tc_lora_tiles(HostState* hs, const PlanView& pv, const moin_p
   CUtensorMap ax, bA, bW, ah, al, bB;
   __nv_bfloat16* hb_lo = hb + (size_t)T * r;   // low parts follow the high parts in the workspace
   moin_status st = make_map(&ax, x, T, d_in, kBM);
-  if (!st) st = make_map(&bA, pool->A, (uint64_t)pool->n_slots * r, d_in, 64);
+  if (!st) st = make_map(&bA, pool->A, (uint64_t)pool->n_slots * r, d_in, r);   // one slot's rows, no neighbours
   if (!st) st = make_map(&ah, hb, T, r, kBM);
   if (!st) st = make_map(&al, hb_lo, T, r, kBM);
   if (!st) st = make_map(&bB, pool->B, (uint64_t)pool->n_slots * d_out, r, 256);
@@ -410,7 +413,7 @@ moin_status launch_tc_lora_tiles(HostState* hs, const PlanView& pv, const moin_p
     ProfScope prof(MOIN_K_SHRINK_TC, 1, stream);
     TcParams p = {};
     p.M = T; p.N = r; p.K = d_in; p.header = pv.header; p.tile_row0 = pv.tile_row0; p.tile_rows = pv.tile_rows;
-    p.tile_expert = pv.tile_expert; p.slot_of_expert = pool->slot_of_expert; p.rows_per_slot = r; p.y = hb; p.y_lo = hb_lo; p.ldy = r;
+    p.tile_expert = pv.tile_expert; p.slot_of_expert = pool->slot_of_expert; p.rows_per_slot = r; p.b_box_rows = r; p.y = hb; p.y_lo = hb_lo; p.ldy = r;
     p.scale = scale; p.status = hs->status;
     st = launch_cfg<64, EPI_SHRINK>(hs, ax, bA, ax, ax, bA, p, max_tiles_m, stream);
     if (st) return st;
