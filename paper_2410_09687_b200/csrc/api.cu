@@ -435,9 +435,24 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
     bool all_tc = true;
     for (int j = 0; j < n_jobs; ++j) all_tc = all_tc && use_tc[j] && tc_fused_supported(r[j]);
     if (all_tc) {
+      // shrinks first: projections with the same d_in and rank share one launch (up to kTcMaxShrinkJobs)
+      for (int j0 = 0; j0 < n_jobs;) {
+        const moin_pool* gp[kTcMaxShrinkJobs];
+        const __nv_bfloat16* gx[kTcMaxShrinkJobs];
+        __nv_bfloat16* gh[kTcMaxShrinkJobs];
+        int n = 0;
+        while (j0 + n < n_jobs && n < kTcMaxShrinkJobs && d_in[j0 + n] == d_in[j0] && r[j0 + n] == r[j0]) {
+          gp[n] = jobs[j0 + n].pool;
+          gx[n] = (const __nv_bfloat16*)jobs[j0 + n].x;
+          gh[n] = reinterpret_cast<__nv_bfloat16*>(ws_job[j0 + n]);
+          ++n;
+        }
+        if ((st = launch_tc_shrink_group(hs, pv, gp, gx, gh, n, scale, s))) return st;
+        j0 += n;
+      }
       for (int j = 0; j < n_jobs; ++j) {
-        st = launch_tc_lora_tiles(hs, pv, jobs[j].pool, (const __nv_bfloat16*)jobs[j].x, (const __nv_bfloat16*)jobs[j].W,
-                                  (__nv_bfloat16*)jobs[j].y, reinterpret_cast<__nv_bfloat16*>(ws_job[j]), scale, s);
+        st = launch_tc_fused(hs, pv, jobs[j].pool, (const __nv_bfloat16*)jobs[j].x, (const __nv_bfloat16*)jobs[j].W,
+                             (__nv_bfloat16*)jobs[j].y, reinterpret_cast<__nv_bfloat16*>(ws_job[j]), s);
         if (st) return st;
       }
       return MOIN_OK;

@@ -30,6 +30,7 @@ constexpr int kBM = 128, kBK = 64;
 constexpr int kTcThreads = 192;
 enum { EPI_STORE = 0, EPI_ROUTER = 1, EPI_SHRINK = 2 };
 
+constexpr int kMaxShrinkJobs = 3;
 struct TcParams {
   int M, N, K;                 // problem: rows, output columns, reduction length
   // plan tiles (nullptr -> regular grid over M)
@@ -47,6 +48,14 @@ struct TcParams {
   float* y0;                   // EPI_STORE: optional fp32 copy
   int ldy;
   float scale;                 // EPI_SHRINK
+  // EPI_SHRINK over several projections that share the plan, K and the rank (n_jobs in 1..kMaxShrinkJobs):
+  // tile index = job * row tiles + row tile; job j reads x through the j-th A-side map and its pool through
+  // the j-th B-side map, looks its slot up in slot_tabs[j] and writes ys[j] / ys_lo[j].  n_jobs = 0: one job
+  // described by slot_of_expert / y / y_lo.
+  int n_jobs;
+  const int* slot_tabs[3];
+  __nv_bfloat16* ys[3];
+  __nv_bfloat16* ys_lo[3];
   const float* inv_norm;       // EPI_ROUTER
   unsigned long long* keys;    // EPI_ROUTER
   DeviceStatus* status;
@@ -85,7 +94,7 @@ template <int BN, int EPI>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmA3,
-               const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
+               const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmB3, const TcParams p) {
   using Cfg = TcCfg<BN>;
   constexpr int S = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
@@ -122,18 +131,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const bool planned = p.header != nullptr;
   const int tiles_n = (p.N + BN - 1) / BN;
   const int tiles_m = planned ? p.header[PH_NTILES] : (p.M + kBM - 1) / kBM;
-  const int total = tiles_m * tiles_n;
+  const int n_jobs = (EPI == EPI_SHRINK && p.n_jobs > 1) ? p.n_jobs : 1;   // EPI_SHRINK: tiles_n == 1
+  const int total = tiles_m * tiles_n * n_jobs;
   const int nkb_main = (p.K + kBK - 1) / kBK;
 
+  int job = 0;   // projection of the current tile (EPI_SHRINK with several jobs), set by tile_info
   auto tile_info = [&](int tile, int& row0, int& rows, int& n0, int& slot) {
-    const int tm = tile / tiles_n;
+    int tm = tile / tiles_n;
     n0 = (tile - tm * tiles_n) * BN;
+    if (EPI == EPI_SHRINK && n_jobs > 1) {
+      job = tm / tiles_m;
+      tm -= job * tiles_m;
+    }
     slot = -1;
     if (planned) {
       row0 = p.tile_row0[tm];
       rows = p.tile_rows[tm];
       const int e = p.tile_expert[tm];
-      if (e >= 0 && p.slot_of_expert) slot = p.slot_of_expert[e];
+      const int* tab = p.slot_of_expert;
+      if (EPI == EPI_SHRINK && p.n_jobs > 0) tab = (job == 0) ? p.slot_tabs[0] : (job == 1) ? p.slot_tabs[1] : p.slot_tabs[2];
+      if (e >= 0 && tab) slot = tab[e];
     } else {
       row0 = tm * kBM;
       rows = min(kBM, p.M - row0);
@@ -158,8 +175,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t b_rows = (kb < nkb_main && p.b_box_rows > 0) ? (uint32_t)p.b_box_rows : (uint32_t)BN;
           mbar_expect_tx(full0 + 8 * s, (kBM + b_rows) * kBK * 2);
           if (kb < nkb_main) {
-            tma_load_2d(sa, &tmA, full0 + 8 * s, kb * kBK, row0);
-            tma_load_2d(sb, &tmB, full0 + 8 * s, kb * kBK, brow);
+            const CUtensorMap* ma = &tmA;
+            const CUtensorMap* mb = &tmB;
+            if (EPI == EPI_SHRINK && job > 0) {
+              ma = (job == 1) ? &tmA2 : &tmA3;
+              mb = (job == 1) ? &tmB2 : &tmB3;
+            }
+            tma_load_2d(sa, ma, full0 + 8 * s, kb * kBK, row0);
+            tma_load_2d(sb, mb, full0 + 8 * s, kb * kBK, brow);
           } else {
             tma_load_2d(sa, kb == nkb_main ? &tmA2 : &tmA3, full0 + 8 * s, 0, row0);
             tma_load_2d(sb, &tmB2, full0 + 8 * s, 0, slot * p.rows_per_slot + n0);
@@ -234,7 +257,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         } else if (row_ok && (EPI == EPI_STORE || slot >= 0)) {
           const float sc = (EPI == EPI_SHRINK) ? p.scale : 1.f;
-          __nv_bfloat16* yrow = p.y + grow * (size_t)p.ldy + n0 + c;
+          __nv_bfloat16* ybase = p.y;
+          __nv_bfloat16* ylo_base = p.y_lo;
+          if (EPI == EPI_SHRINK && p.n_jobs > 0) {
+            ybase = (job == 0) ? p.ys[0] : (job == 1) ? p.ys[1] : p.ys[2];
+            ylo_base = (job == 0) ? p.ys_lo[0] : (job == 1) ? p.ys_lo[1] : p.ys_lo[2];
+          }
+          __nv_bfloat16* yrow = ybase + grow * (size_t)p.ldy + n0 + c;
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
             if (n0 + c + j < p.N) {  // N is a multiple of 8
@@ -253,7 +282,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 l.y = pack_bf16(f[2] - bf16_lo(o.y), f[3] - bf16_hi(o.y));
                 l.z = pack_bf16(f[4] - bf16_lo(o.z), f[5] - bf16_hi(o.z));
                 l.w = pack_bf16(f[6] - bf16_lo(o.w), f[7] - bf16_hi(o.w));
-                *reinterpret_cast<uint4*>(p.y_lo + grow * (size_t)p.ldy + n0 + c + j) = l;
+                *reinterpret_cast<uint4*>(ylo_base + grow * (size_t)p.ldy + n0 + c + j) = l;
               }
               if (EPI == EPI_STORE && p.y0) {
                 float* y0row = p.y0 + grow * (size_t)p.ldy + n0 + c + j;
@@ -325,7 +354,7 @@ moin_status make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t
 template <int BN, int EPI>
 static moin_status launch_cfg(HostState* hs, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& a2,
                               const CUtensorMap& a3, const CUtensorMap& b2, const TcParams& p, long max_tiles,
-                              cudaStream_t stream) {
+                              cudaStream_t stream, const CUtensorMap* b3 = nullptr) {
   using Cfg = TcCfg<BN>;
   static bool configured = false;
   if (!configured) {
@@ -336,7 +365,7 @@ static moin_status launch_cfg(HostState* hs, const CUtensorMap& a, const CUtenso
   }
   long grid = max_tiles < hs->n_sms ? max_tiles : hs->n_sms;
   if (grid < 1) grid = 1;
-  tc_gemm_kernel<BN, EPI><<<(int)grid, kTcThreads, Cfg::kSmemBytes, stream>>>(a, b, a2, a3, b2, p);
+  tc_gemm_kernel<BN, EPI><<<(int)grid, kTcThreads, Cfg::kSmemBytes, stream>>>(a, b, a2, a3, b2, b3 ? *b3 : b2, p);
   return record_cuda(cudaGetLastError());
 }
 
@@ -394,36 +423,53 @@ moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_b
   return launch_cfg<64, EPI_ROUTER>(hs, a, b, a, a, b, p, tiles, stream);
 }
 
-moin_status launch_tc_lora_tiles(HostState* hs, const PlanView& pv, const moin_pool* pool, const __nv_bfloat16* x,
-                                 const __nv_bfloat16* W, __nv_bfloat16* y, __nv_bfloat16* hb, float scale,
-                                 cudaStream_t stream) {
-  const int T = pv.T, d_in = pool->d_in, d_out = pool->d_out, r = pool->r;
-  // upper bound on row tiles without reading the plan back: every run adds at most one partial tile
-  const long max_tiles_m = T;  // grid is capped at the SM count; the kernel reads the true count
-  CUtensorMap ax, bA, bW, ah, al, bB;
-  __nv_bfloat16* hb_lo = hb + (size_t)T * r;   // low parts follow the high parts in the workspace
-  moin_status st = make_map(&ax, x, T, d_in, kBM);
-  if (!st) st = make_map(&bA, pool->A, (uint64_t)pool->n_slots * r, d_in, r);   // one slot's rows, no neighbours
-  if (!st) st = make_map(&ah, hb, T, r, kBM);
-  if (!st) st = make_map(&al, hb_lo, T, r, kBM);
-  if (!st) st = make_map(&bB, pool->B, (uint64_t)pool->n_slots * d_out, r, 256);
-  if (st) return st;
-  // 1. hb[row, :r] = bf16(scale * x A_e^T)   (one N tile of 64 columns, rank columns stored)
-  {
-    ProfScope prof(MOIN_K_SHRINK_TC, 1, stream);
-    TcParams p = {};
-    p.M = T; p.N = r; p.K = d_in; p.header = pv.header; p.tile_row0 = pv.tile_row0; p.tile_rows = pv.tile_rows;
-    p.tile_expert = pv.tile_expert; p.slot_of_expert = pool->slot_of_expert; p.rows_per_slot = r; p.b_box_rows = r; p.y = hb; p.y_lo = hb_lo; p.ldy = r;
-    p.scale = scale; p.status = hs->status;
-    st = launch_cfg<64, EPI_SHRINK>(hs, ax, bA, ax, ax, bA, p, max_tiles_m, stream);
+// Long-run mode, step 1 for up to kMaxShrinkJobs projections that share the plan, d_in and the rank:
+// hb_j[row, :r] = hi/lo bf16 parts of scale * x_j A_j,e^T in ONE launch (row tiles of all the projections in
+// one persistent grid, so set-up, first round trip and tail are paid once).
+moin_status launch_tc_shrink_group(HostState* hs, const PlanView& pv, const moin_pool* const* pools,
+                                   const __nv_bfloat16* const* xs, __nv_bfloat16* const* hbs, int n_jobs, float scale,
+                                   cudaStream_t stream) {
+  if (n_jobs < 1 || n_jobs > kMaxShrinkJobs) return MOIN_ERR_INVALID_ARG;
+  const int T = pv.T, d_in = pools[0]->d_in, r = pools[0]->r;
+  CUtensorMap ax[kMaxShrinkJobs], bA[kMaxShrinkJobs];
+  TcParams p = {};
+  p.M = T; p.N = r; p.K = d_in; p.header = pv.header; p.tile_row0 = pv.tile_row0; p.tile_rows = pv.tile_rows;
+  p.tile_expert = pv.tile_expert; p.rows_per_slot = r; p.b_box_rows = r; p.ldy = r;
+  p.scale = scale; p.status = hs->status; p.n_jobs = n_jobs;
+  for (int j = 0; j < n_jobs; ++j) {
+    if (pools[j]->d_in != d_in || pools[j]->r != r) return MOIN_ERR_INVALID_ARG;
+    moin_status st = make_map(&ax[j], xs[j], T, d_in, kBM);
+    if (!st) st = make_map(&bA[j], pools[j]->A, (uint64_t)pools[j]->n_slots * r, d_in, r);   // one slot's rows, no neighbours
     if (st) return st;
+    p.slot_tabs[j] = pools[j]->slot_of_expert;
+    p.ys[j] = hbs[j];
+    p.ys_lo[j] = hbs[j] + (size_t)T * r;   // low parts follow the high parts in the workspace
   }
-  // 2. y = [x | hb] [W ; B_e]^T
+  for (int j = n_jobs; j < kMaxShrinkJobs; ++j) {   // unused maps: any valid one
+    ax[j] = ax[0];
+    bA[j] = bA[0];
+  }
+  ProfScope prof(MOIN_K_SHRINK_TC, 1, stream);
+  // upper bound on row tiles without reading the plan back: every run adds at most one partial tile;
+  // the grid is capped at the SM count and the kernel reads the true count
+  return launch_cfg<64, EPI_SHRINK>(hs, ax[0], bA[0], ax[1], ax[2], bA[1], p, (long)T * n_jobs, stream, &bA[2]);
+}
+
+// Long-run mode, step 2: y = [x | hi | lo] [W ; B_e ; B_e]^T with hb from step 1.
+moin_status launch_tc_fused(HostState* hs, const PlanView& pv, const moin_pool* pool, const __nv_bfloat16* x,
+                            const __nv_bfloat16* W, __nv_bfloat16* y, __nv_bfloat16* hb, cudaStream_t stream) {
+  const int T = pv.T, d_in = pool->d_in, d_out = pool->d_out, r = pool->r;
+  const long max_tiles_m = T;
+  CUtensorMap ax, bW, ah, al, bB;
+  __nv_bfloat16* hb_lo = hb + (size_t)T * r;
   ProfScope prof(MOIN_K_FUSED_TC, 1, stream);
   const long full_tiles_m = (T + kBM - 1) / kBM;
   const int bn = pick_bn(full_tiles_m, d_out, hs->n_sms);
-  st = make_map(&bW, W, d_out, d_in, bn);
-  if (!st && bn != 256) st = make_map(&bB, pool->B, (uint64_t)pool->n_slots * d_out, r, bn);
+  moin_status st = make_map(&ax, x, T, d_in, kBM);
+  if (!st) st = make_map(&ah, hb, T, r, kBM);
+  if (!st) st = make_map(&al, hb_lo, T, r, kBM);
+  if (!st) st = make_map(&bW, W, d_out, d_in, bn);
+  if (!st) st = make_map(&bB, pool->B, (uint64_t)pool->n_slots * d_out, r, bn);
   if (st) return st;
   TcParams p = {};
   p.M = T; p.N = d_out; p.K = d_in; p.header = pv.header; p.tile_row0 = pv.tile_row0; p.tile_rows = pv.tile_rows;

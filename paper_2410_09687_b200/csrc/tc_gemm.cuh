@@ -23,9 +23,12 @@ moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_b
                              int Q, int K, int D, unsigned long long* keys, cudaStream_t stream);
 // Tile mode: hb = hi/lo bf16 parts of s * x A_e^T per row tile ([2][T][r]), then y = [x | hi | lo] [W ; B_e ; B_e]^T
 // in one GEMM.
-moin_status launch_tc_lora_tiles(HostState* hs, const PlanView& pv, const moin_pool* pool, const __nv_bfloat16* x,
-                                 const __nv_bfloat16* W, __nv_bfloat16* y, __nv_bfloat16* hb, float scale,
-                                 cudaStream_t stream);
+moin_status launch_tc_shrink_group(HostState* hs, const PlanView& pv, const moin_pool* const* pools,
+                                   const __nv_bfloat16* const* xs, __nv_bfloat16* const* hbs, int n_jobs, float scale,
+                                   cudaStream_t stream);
+constexpr int kTcMaxShrinkJobs = 3;   // projections one grouped shrink launch can take
+moin_status launch_tc_fused(HostState* hs, const PlanView& pv, const moin_pool* pool, const __nv_bfloat16* x,
+                            const __nv_bfloat16* W, __nv_bfloat16* y, __nv_bfloat16* hb, cudaStream_t stream);
 
 // TMA-staged segmented LoRA kernels (short segments), up to 4 projections per launch.  The shrink writes
 // lora_stream_parts(d_in) partial results hpart[part][T][r] per projection; the expand sums them in index order.
