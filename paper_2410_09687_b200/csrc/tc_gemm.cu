@@ -369,11 +369,21 @@ static moin_status launch_cfg(HostState* hs, const CUtensorMap& a, const CUtenso
   return record_cuda(cudaGetLastError());
 }
 
+// Tile width for many row tiles: the one with the least (waves of tiles over the SMs) x (time of one tile), a
+// tile's time taken as proportional to BN plus a fixed part worth 64 columns.  A projection as narrow as k or v
+// (N = 256) then runs as one wave of 128 x 256 tiles rather than two of 128 x 128.
 static int pick_bn(long tiles_m, int N, int n_sms) {
-  for (int bn : {256, 128}) {
-    if (tiles_m * ((N + bn - 1) / bn) >= n_sms) return bn;
+  int best = 64;
+  long best_cost = -1;
+  for (int bn : {256, 128, 64}) {
+    const long tiles = tiles_m * ((N + bn - 1) / bn);
+    const long cost = ((tiles + n_sms - 1) / n_sms) * (bn + 64);
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best = bn;
+    }
   }
-  return 64;
+  return best;
 }
 // Few row tiles (decode): a CTA's duration grows with the bytes it pulls, (128 + BN) * K * 2.  This GEMM runs
 // beside the adapter shrink and the expand waits for both, so take the widest tile (fewest CTAs, least
