@@ -108,7 +108,7 @@ class ClockSampler:
 class LayerWorkload:
     """route -> plan -> seven projections.  decode: E=500 r=64 T=256; prefill: E=5000 r=16 32x512."""
 
-    def __init__(self, kind: str, dev: str, grouped: bool = True):
+    def __init__(self, kind: str, dev: str, grouped: bool = True, rank=None):
         import paper_2410_09687_b200 as moin
         self.moin, self.kind, self.dev, self.grouped = moin, kind, dev, grouped
         if kind == "decode":
@@ -117,6 +117,8 @@ class LayerWorkload:
         else:
             self.E, self.r, self.T, self.R, self.K, self.seed = 5000, 16, 16384, 32, 5000, 2
             self.mode = moin.PLAN_TILES
+        if rank:   # side measurement at another rank (the paper trains its experts at 128, Sec. 4)
+            self.r = int(rank)
         self.D, self.scale = 768, 2.0
         self.unit, self.units_per_step = "tokens", self.T
         self.projs = mi.TINYLLAMA_PROJECTIONS
@@ -215,9 +217,9 @@ class LayerWorkload:
         return {"per_kernel_bytes": per, "step_bytes": step_bytes, "step_flops": flops}
 
     def config(self) -> dict:
-        name = ("decode: 7 TinyLlama projections, 500 experts rank 64, 256 single tokens, router 256x500x768"
+        name = (f"decode: 7 TinyLlama projections, 500 experts rank {self.r}, 256 single tokens, router 256x500x768"
                 if self.kind == "decode" else
-                "prefill: 7 TinyLlama projections, 5000 experts rank 16, 32x512 tokens Zipf(1.1), router 32x5000x768")
+                f"prefill: 7 TinyLlama projections, 5000 experts rank {self.r}, 32x512 tokens Zipf(1.1), router 32x5000x768")
         return {"workload": name, "calls": ("grouped {q,k,v} {o} {gate,up} {down}" if self.grouped else "one call per projection"),
                 "tokens_per_step": self.T, "experts": self.E, "rank": self.r, "lora_scale": self.scale,
                 "l2": f"inputs rotate over {ROTATE} batches; per-step working set exceeds L2"}
@@ -525,6 +527,7 @@ def main():
     ap.add_argument("--no-router-extra", action="store_true")
     ap.add_argument("--forward-layers", type=int, default=22)
     ap.add_argument("--no-group", action="store_true", help="one moin_lora_linear call per projection")
+    ap.add_argument("--rank", type=int, default=None, help="decode / prefill at another LoRA rank than the config's (side measurement)")
     ap.add_argument("--stream-impl", type=int, default=0, help="short-segment LoRA kernels: 0 auto, 1 register-fed, 2 TMA-staged")
     args = ap.parse_args()
     defaults = {"decode": (3000, 20), "prefill": (100, 5), "router": (50, 5), "forward": (5, 3)}
@@ -550,7 +553,7 @@ def main():
     peaks = load_peaks()
     kind = args.workload
     if kind in ("decode", "prefill"):
-        wl = LayerWorkload(kind, dev, grouped=not args.no_group)
+        wl = LayerWorkload(kind, dev, grouped=not args.no_group, rank=args.rank)
     elif kind == "router":
         wl = RouterWorkload(dev)
     else:

@@ -49,7 +49,7 @@ enum {
   MOIN_ERR_BAD_SHAPE = -2,        /* a dimension violates the documented divisibility rules */
   MOIN_ERR_MISALIGNED = -3,       /* a tensor pointer is not 16-byte aligned */
   MOIN_ERR_WORKSPACE = -4,        /* workspace too small or null */
-  MOIN_ERR_UNSUPPORTED_RANK = -5, /* LoRA rank not a multiple of 8 in 8..64 */
+  MOIN_ERR_UNSUPPORTED_RANK = -5, /* LoRA rank not a multiple of 8 in 8..128 */
   MOIN_ERR_CUDA = -6,             /* a CUDA runtime/driver call failed (see moin_last_cuda_error) */
   MOIN_ERR_TIMEOUT = -7,          /* a device-side bounded wait ran out (reported by moin_device_status) */
   MOIN_ERR_NO_DEVICE = -8         /* no sm_100 device is current */
@@ -163,7 +163,7 @@ typedef struct {
   const int32_t* slot_of_expert; /* [E] int32, values in [-1, n_slots) */
   int32_t E;
   int32_t n_slots;
-  int32_t r;     /* LoRA rank: multiple of 8, 8..64 */
+  int32_t r;     /* LoRA rank: multiple of 8, 8..128 (128 is the rank of the paper's experts, Sec. 4) */
   int32_t d_in;  /* multiple of 64 */
   int32_t d_out; /* multiple of 8 */
 } moin_pool;

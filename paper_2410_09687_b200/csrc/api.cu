@@ -356,7 +356,7 @@ size_t moin_lora_linear_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, 
   const size_t parts = (size_t)lora_stream_parts(d_in > 0 ? d_in : 64);
   size_t seg = align_up(parts * (size_t)T * (size_t)(r > 0 ? r : 8) * sizeof(float), 256) +
                align_up((size_t)T * (size_t)d_out * sizeof(float), 256);
-  size_t tiles = align_up(2 * Tp * (size_t)64 * sizeof(__nv_bfloat16), 256);   // hi and lo parts of s * (x A^T)
+  size_t tiles = align_up(2 * Tp * (size_t)(r > 64 ? r : 64) * sizeof(__nv_bfloat16), 256);   // hi and lo parts of s * (x A^T)
   return (seg > tiles ? seg : tiles) + 256;
 }
 
@@ -375,7 +375,7 @@ static moin_status check_job(const moin_plan* plan, const void* x, const void* W
   if (!aligned16(x) || !aligned16(W) || !aligned16(y)) return MOIN_ERR_MISALIGNED;
   if (lora) {
     *r = pool->r;
-    if (*r < 8 || *r > 64 || (*r % 8) != 0) return MOIN_ERR_UNSUPPORTED_RANK;
+    if (*r < 8 || *r > 128 || (*r % 8) != 0) return MOIN_ERR_UNSUPPORTED_RANK;
     if (!pool->A || !pool->B || !pool->slot_of_expert || !plan->buffer) return MOIN_ERR_INVALID_ARG;
     if (pool->E != plan->E) return MOIN_ERR_INVALID_ARG;
     if (!aligned16(pool->A) || !aligned16(pool->B)) return MOIN_ERR_MISALIGNED;
@@ -466,7 +466,7 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
   float* y0[kMaxStreamJobs];
   int parts[kMaxStreamJobs];
   bool tma_stream = hs->stream_impl == 2;   // MOIN_OPT_STREAM_IMPL: TMA-staged kernels
-  for (int j = 0; j < n_jobs; ++j) tma_stream = tma_stream && lora_shrink_tma_supported(d_in[j]);
+  for (int j = 0; j < n_jobs; ++j) tma_stream = tma_stream && lora_shrink_tma_supported(d_in[j]) && r[j] <= 64;
   int* queue = reinterpret_cast<int*>(ws_job[0] + moin_lora_linear_workspace_bytes(T, d_in[0], d_out[0], r[0]) - 256);
   const moin_pool* pools[kMaxStreamJobs];
   const __nv_bfloat16* xs[kMaxStreamJobs];

@@ -169,7 +169,7 @@ template <int P>  // number of 32-wide rho groups: ceil(max r / 32)
 __global__ void __launch_bounds__(kExpandThreads, 4)
 lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict__ perm,
                           const int4* __restrict__ seg_tab, const ExpandJobs jobs, float scale, int tps) {
-  constexpr int TB = kExpandTilesPerBatch;
+  constexpr int TB = P > 2 ? 1 : kExpandTilesPerBatch;   // wide ranks: one tile's rows already fill the load registers
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const long long wid = (long long)blockIdx.x * (kExpandThreads / 32) + warp;
@@ -321,8 +321,10 @@ cudaError_t launch_lora_expand_stream(const PlanView& pv, ExpandJobs jobs, float
   const int grid = stream_grid(max_ctas, n_sms, 4);
   if (rmax <= 32)
     lora_expand_stream_kernel<1><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale, tps);
-  else
+  else if (rmax <= 64)
     lora_expand_stream_kernel<2><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale, tps);
+  else
+    lora_expand_stream_kernel<4><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale, tps);
   return cudaGetLastError();
 }
 

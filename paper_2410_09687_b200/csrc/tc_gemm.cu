@@ -166,7 +166,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int row0, rows, n0, slot;
         tile_info(tile, row0, rows, n0, slot);
         const bool tail = (EPI == EPI_STORE) && planned && p.tail_r > 0 && slot >= 0;
-        const int nkb = nkb_main + (tail ? 2 : 0);   // tail: [hi(s h) | lo(s h)] x [B_e ; B_e]
+        const int nrb = (p.tail_r + kBK - 1) / kBK;   // 64-wide blocks of the rank
+        const int nkb = nkb_main + (tail ? 2 * nrb : 0);   // tail: [hi(s h) | lo(s h)] x [B_e ; B_e], nrb blocks each
         const int brow = (EPI == EPI_SHRINK) ? (slot >= 0 ? slot : 0) * p.rows_per_slot : n0;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const uint32_t s = it % S, ph = (it / S) & 1u;
@@ -184,8 +185,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tma_load_2d(sa, ma, full0 + 8 * s, kb * kBK, row0);
             tma_load_2d(sb, mb, full0 + 8 * s, kb * kBK, brow);
           } else {
-            tma_load_2d(sa, kb == nkb_main ? &tmA2 : &tmA3, full0 + 8 * s, 0, row0);
-            tma_load_2d(sb, &tmB2, full0 + 8 * s, 0, slot * p.rows_per_slot + n0);
+            const int j = kb - nkb_main, rb = (j >= nrb) ? j - nrb : j;   // hi blocks first, then lo blocks
+            tma_load_2d(sa, j < nrb ? &tmA2 : &tmA3, full0 + 8 * s, rb * kBK, row0);
+            tma_load_2d(sb, &tmB2, full0 + 8 * s, rb * kBK, slot * p.rows_per_slot + n0);
           }
         }
       }
@@ -200,7 +202,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int row0, rows, n0, slot;
         tile_info(tile, row0, rows, n0, slot);
         const bool tail = (EPI == EPI_STORE) && planned && p.tail_r > 0 && slot >= 0;
-        const int nkb = nkb_main + (tail ? 2 : 0);
+        const int nrb = (p.tail_r + kBK - 1) / kBK;
+        const int nkb = nkb_main + (tail ? 2 * nrb : 0);
         const uint32_t acc = lt & 1u, aph = (lt >> 1) & 1u;
         if (!(ok = mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag, p.status, 2))) break;
         tc_fence_after();
@@ -211,7 +214,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tc_fence_after();
           const uint32_t sa = tiles_base + s * Cfg::kStageBytes, sb = sa + kBM * kBK * 2;
           const uint64_t da = make_sdesc(sa), db = make_sdesc(sb);
-          const int nk16 = (kb < nkb_main) ? (min(kBK, p.K - kb * kBK) + 15) / 16 : (p.tail_r + 15) / 16;
+          int nk16 = (min(kBK, p.K - kb * kBK) + 15) / 16;
+          if (kb >= nkb_main) {
+            const int j = kb - nkb_main, rb = (j >= nrb) ? j - nrb : j;
+            nk16 = (min(kBK, p.tail_r - rb * kBK) + 15) / 16;
+          }
           for (int k = 0; k < nk16; ++k)
             tc_mma_bf16(tmem_d, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb > 0 || k > 0) ? 1u : 0u);
           tc_commit(empty0 + 8 * s);
@@ -399,7 +406,7 @@ static int pick_bn_small_m(int N, int K) {
 
 bool tc_gemm_supported(int T, int d_in, int d_out) { return T >= 1 && d_in >= 64 && (d_in % 8) == 0 && (d_out % 8) == 0; }
 bool tc_router_supported(int Q, int K, int D) { return Q >= 1 && K >= 1 && D >= 64 && (D % 8) == 0; }
-bool tc_fused_supported(int r) { return r >= 8 && r <= 64 && (r % 8) == 0; }
+bool tc_fused_supported(int r) { return r >= 8 && r <= 128 && (r % 8) == 0; }
 
 moin_status launch_tc_gemm(HostState* hs, const __nv_bfloat16* x, const __nv_bfloat16* W, __nv_bfloat16* y, float* y0,
                            int T, int d_in, int d_out, cudaStream_t stream) {
@@ -462,6 +469,7 @@ moin_status launch_tc_shrink_group(HostState* hs, const PlanView& pv, const moin
   ProfScope prof(MOIN_K_SHRINK_TC, 1, stream);
   // upper bound on row tiles without reading the plan back: every run adds at most one partial tile;
   // the grid is capped at the SM count and the kernel reads the true count
+  if (r > 64) return launch_cfg<128, EPI_SHRINK>(hs, ax[0], bA[0], ax[1], ax[2], bA[1], p, (long)T * n_jobs, stream, &bA[2]);
   return launch_cfg<64, EPI_SHRINK>(hs, ax[0], bA[0], ax[1], ax[2], bA[1], p, (long)T * n_jobs, stream, &bA[2]);
 }
 

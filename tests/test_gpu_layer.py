@@ -45,7 +45,7 @@ def stream_impl(request):
     moin.set_option(moin.OPT_STREAM_IMPL, 0)
 
 
-@pytest.mark.parametrize("r", [8, 16, 24, 32, 40, 48, 56, 64])
+@pytest.mark.parametrize("r", [8, 16, 24, 32, 40, 48, 56, 64, 72, 96, 120, 128])
 @pytest.mark.parametrize("mode", MODES)
 def test_every_supported_rank(r, mode, stream_impl):
     rng = mi.np_rng(7, r)
@@ -74,6 +74,27 @@ def test_base_only_and_missing_adapters(mode, stream_impl):
     assert torch.equal(y[torch.from_numpy(base_rows).to(DEV)], y_base[torch.from_numpy(base_rows).to(DEV)])
     assert_layer_close(y_base, oracle.lora_linear(mi.bf16_bits(case.x), mi.bf16_bits(case.W), None, None, None,
                                                   None, 0.0), "base")
+
+
+def test_decode_shape_at_the_papers_rank_128():
+    # Sec. 4 trains every expert at rank 128: 256 single-token requests over 120 such experts, a wide projection
+    E, r, T, d_in, d_out = 120, 128, 256, 2048, 2048
+    pool = mi.make_pool(E, r, d_in, d_out, 21, 1)
+    te = mi.np_rng(21, 2).integers(0, E, size=T).astype(np.int32)
+    case = mi.layer_case("rank128", T, d_in, d_out, pool, te, 2.0, 21, 3)
+    y, _ = run_layer(case, moin.PLAN_SEGMENTS)
+    assert_layer_close(y, oracle_layer(case), "rank 128 decode")
+
+
+def test_long_runs_at_rank_128_through_the_fused_gemm():
+    # 8 requests x 256 tokens, full-width projection: the rank spans two 64-wide blocks of the appended K range
+    E, r, d_in, d_out = 16, 128, 2048, 2048
+    pool = mi.make_pool(E, r, d_in, d_out, 22, 1, missing=(5,))
+    req = np.array([3, 7, 5, 0, -1, 15, 7, 2], np.int32)
+    te = np.repeat(req, 256).astype(np.int32)
+    case = mi.layer_case("rank128 runs", len(te), d_in, d_out, pool, te, 2.0, 22, 3)
+    y, _ = run_layer(case, moin.PLAN_TILES)
+    assert_layer_close(y, oracle_layer(case), "rank 128 long runs")
 
 
 def test_decode_config_all_projections(stream_impl):
