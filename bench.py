@@ -338,15 +338,20 @@ class ForwardWorkload:
 # ----------------------------------------------------------------------------------------------
 # measurement helpers
 # ----------------------------------------------------------------------------------------------
-def dist_setup(n_gpus: int):
+def dist_setup(n_gpus: int, backend: str = "nccl"):
+    """One process per GPU (replicas): reads RANK / LOCAL_RANK / WORLD_SIZE; the process group only carries the
+    barrier and the max-over-ranks of the timing.  `backend="gloo"` runs the same logic on CPU (tests)."""
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if world > 1:
         import torch.distributed as dist
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    else:
+        if backend == "nccl":
+            torch.cuda.set_device(local)
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(backend)
+    elif backend == "nccl":
         torch.cuda.set_device(0)
         local = 0
     return world, rank, local
@@ -361,10 +366,17 @@ def barrier(world):
 def max_over_ranks(world, v: float) -> float:
     if world > 1:
         import torch.distributed as dist
-        t = torch.tensor([v], dtype=torch.float64, device="cuda")
+        dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+        t = torch.tensor([v], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
     return v
+
+
+def whole_job_value(world: int, units_per_step: float, ms_per_step_max: float) -> float:
+    """Aggregate throughput of `world` replicas that each process units_per_step per step (weak scaling):
+    all the units divided by the slowest rank's time."""
+    return world * units_per_step / (ms_per_step_max * 1e-3)
 
 
 def timed_loop(world, fn, steps: int, warmup: int, use_graph: bool) -> float:
@@ -566,7 +578,7 @@ def main():
     ms, graphed = timed_loop(world, wl.step, args.steps, args.warmup, use_graph)
     clocks = sampler.stop()
     ms = max_over_ranks(world, ms)
-    value = world * wl.units_per_step / (ms * 1e-3)
+    value = whole_job_value(world, wl.units_per_step, ms)
 
     e2e_steps = max(5, args.steps // 4)
     ms_e2e, _ = timed_loop(world, wl.step_e2e, e2e_steps, max(3, args.warmup // 2), use_graph)
@@ -673,7 +685,7 @@ def main():
         line = {"metric": metric, "value": value, "unit": wl.unit + "/s", "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": cfg, "clocks": clocks,
-                "e2e": {"value": world * wl.units_per_step / (ms_e2e * 1e-3), "unit": wl.unit + "/s",
+                "e2e": {"value": whole_job_value(world, wl.units_per_step, ms_e2e), "unit": wl.unit + "/s",
                         "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "ms_per_step": ms_e2e},
                 "gpu_launches": int(round(launches_per_step * args.steps)), "roofline": roof, "kernels": kernels,
                 "cpu_baseline": cpu}
