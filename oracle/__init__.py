@@ -70,6 +70,10 @@ def lib() -> ctypes.CDLL:
         L.moin_oracle_bucket.restype = ctypes.c_int64
         L.moin_oracle_bucket.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                          ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        L.moin_oracle_kmeans_update.restype = ctypes.c_int
+        L.moin_oracle_kmeans_update.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
+                                                ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
+                                                ctypes.c_void_p]
         _lib = L
     return _lib
 
@@ -165,6 +169,22 @@ def bucket(token_expert: np.ndarray, slot_of_expert: np.ndarray, n_slots: int) -
     if S < 0:
         raise RuntimeError("moin_oracle_bucket failed")
     return {"perm": perm[:T], "seg_slot": seg_slot[:S], "seg_start": seg_start[:S + 1], "S": int(S)}
+
+
+def kmeans_update(x: np.ndarray, c_old: np.ndarray, assign: np.ndarray) -> Dict[str, np.ndarray]:
+    """K-means update step: mean of every cluster's members (float64); empty clusters keep c_old's row."""
+    (x, c_old), kind = _same_kind(x, c_old)
+    N, D = x.shape
+    K = c_old.shape[0]
+    assert c_old.shape[1] == D
+    a = np.ascontiguousarray(assign, dtype=np.int32)
+    assert a.shape == (N,)
+    c_new = np.zeros((K, D), np.float64)
+    counts = np.zeros(K, np.int64)
+    rc = lib().moin_oracle_kmeans_update(_ptr(x), _ptr(c_old), kind, _ptr(a), N, K, D, _ptr(c_new), _ptr(counts))
+    if rc:
+        raise RuntimeError(f"moin_oracle_kmeans_update failed: {rc}")
+    return {"centroids": c_new, "counts": counts}
 
 
 PROJ_ORDER = ("q", "k", "v", "o", "gate", "up", "down")

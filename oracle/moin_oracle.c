@@ -10,7 +10,9 @@
  *     token (one expert per request, Sec. 3.3), an optional scale s on the low-rank term
  *     and "no adapter => base model only" (Sec. 4, downstream-task paragraph);
  *   - a Llama-architecture decoder forward (Sec. 4 names the base model) in which every one
- *     of the seven per-block projections is that layer.
+ *     of the seven per-block projections is that layer;
+ *   - the update step of the K-means clustering of document embeddings whose centroids are
+ *     the topic embeddings the router searches (Sec. 3.1, second approach; Sec. 4).
  *
  * No blocking, no fusion, no reordering: every sum runs over its index in increasing
  * order.  Parallelism (OpenMP) is only over independent units: queries, tokens, requests.
@@ -413,4 +415,33 @@ int64_t moin_oracle_bucket(const int32_t* token_expert, const int32_t* slot_of_e
     if (s < 0 || s >= n_slots) perm[pos++] = (int32_t)t;
   }
   return S;
+}
+
+/* ---------------------------------------------------------------------------------------
+ * K-means update (Sec. 3.1: K-means directly in the document embedding space; Sec. 4: the
+ * cluster centroid is the topic embedding).  Given the assignment of every point, centroid
+ * k becomes the arithmetic mean of its members, summed in increasing point order.
+ * Readings: a cluster without members keeps its previous centroid; assignments outside
+ * [0, K) are ignored.  The assignment step itself is the router above (nearest centroid
+ * under the cosine metric), so one Lloyd iteration = route, then this.
+ *
+ * x [N, D], c_old [K, D] (double or bf16 bits); assign [N]; c_new [K, D] double; counts [K].
+ * ------------------------------------------------------------------------------------ */
+int moin_oracle_kmeans_update(const void* x, const void* c_old, int dtype, const int32_t* assign,
+                              int64_t N, int64_t K, int64_t D, double* c_new, int64_t* counts) {
+  if (N < 0 || K < 1 || D < 1) return -1;
+  for (int64_t k = 0; k < K; ++k) counts[k] = 0;
+  for (int64_t i = 0; i < K * D; ++i) c_new[i] = 0.0;
+  for (int64_t i = 0; i < N; ++i) {
+    const int64_t k = assign[i];
+    if (k < 0 || k >= K) continue;
+    counts[k] += 1;
+    for (int64_t d = 0; d < D; ++d) c_new[k * D + d] += ld(x, dtype, (size_t)(i * D + d));
+  }
+  for (int64_t k = 0; k < K; ++k)
+    for (int64_t d = 0; d < D; ++d) {
+      if (counts[k] > 0) c_new[k * D + d] /= (double)counts[k];
+      else c_new[k * D + d] = ld(c_old, dtype, (size_t)(k * D + d));
+    }
+  return 0;
 }
