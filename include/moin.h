@@ -93,7 +93,7 @@ typedef struct {
 enum {
   MOIN_K_ROUTE_SIMPLE = 0, MOIN_K_ROUTE_TC = 1, MOIN_K_ROUTE_FINISH = 2, MOIN_K_PLAN = 3, MOIN_K_GEMM_WARP = 4,
   MOIN_K_GEMM_TC = 5, MOIN_K_SHRINK_STREAM = 6, MOIN_K_EXPAND_STREAM = 7, MOIN_K_SHRINK_TC = 8,
-  MOIN_K_FUSED_TC = 9, MOIN_K_GLUE = 10, MOIN_K_ATTENTION = 11, MOIN_K_ROUTE_CLUSTER = 12, MOIN_K_COUNT = 13
+  MOIN_K_FUSED_TC = 9, MOIN_K_GLUE = 10, MOIN_K_ATTENTION = 11, MOIN_K_ROUTE_CLUSTER = 12, MOIN_K_KMEANS_UPDATE = 13, MOIN_K_COUNT = 14
 };
 moin_status moin_profile_enable(int32_t capacity);
 moin_status moin_profile_read(moin_profile_record* out, int32_t capacity, int32_t* n);
@@ -206,6 +206,26 @@ moin_status moin_plan_build(const int32_t* token_expert, moin_plan* plan, moin_s
 moin_status moin_plan_read(const moin_plan* plan, int32_t* n_segments, int32_t* n_tiles, int32_t* perm,
                            int32_t* seg_expert, int32_t* seg_start, int32_t* tile_row0, int32_t* tile_rows,
                            int32_t* tile_expert, moin_stream stream);
+
+/* ---------------------------------------------------------------------------------------
+ * K-means update.  Paper Sec. 3.1 (second approach): the topics are a K-means clustering of the
+ * document embeddings; Sec. 4: the cluster centroid is the topic embedding the router searches.
+ * One Lloyd iteration over N points is moin_route (assignment: nearest centroid under the cosine
+ * metric), moin_plan_build on the N assignments with E = K (grouping of the points by cluster),
+ * then this call: centroid k <- arithmetic mean of its members, summed in increasing point order
+ * in fp32 and rounded once to bf16.  A cluster without members keeps its previous centroid;
+ * points whose assignment is outside [0, K) belong to no cluster.
+ *
+ *   plan           built from the assignments (plan->T = N points, plan->E = K clusters), any mode
+ *   x              device, [N, D] bf16 row-major, 16-byte aligned; D a multiple of 8, 8..8192
+ *   centroids_old  device, [K, D] bf16; centroids_new device, [K, D] bf16 (may be the same buffer)
+ *   inv_norm_new   device, [K] fp32 or NULL: 1/|c_k| of the NEW (bf16-rounded) centroids, 0 for a zero
+ *                  row, i.e. what moin_router_prepare would compute for them
+ * Asynchronous on `stream`; borrows everything, allocates nothing.  Errors: INVALID_ARG, BAD_SHAPE,
+ * MISALIGNED; launches nothing on error.  N = 0 only copies the centroids. */
+moin_status moin_kmeans_update(const moin_plan* plan, const void* x, const void* centroids_old, void* centroids_new,
+                               float* inv_norm_new, int32_t D, moin_stream stream);
+
 
 /* ---------------------------------------------------------------------------------------
  * Routed LoRA linear layer.  Paper Sec. 3.2: y = W x + W_b (W_a x), W in R^{k x d}; the

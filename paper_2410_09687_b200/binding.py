@@ -23,6 +23,7 @@ EXPORTED_SYMBOLS = (
     "moin_plan_build", "moin_plan_read", "moin_lora_linear_workspace_bytes", "moin_lora_linear",
     "moin_decoder_workspace_bytes", "moin_decoder_forward", "moin_profile_enable", "moin_profile_read",
     "moin_kernel_name", "moin_route_static", "moin_lora_linear_group", "moin_lora_linear_group_workspace_bytes",
+    "moin_kmeans_update",
 )
 
 
@@ -98,6 +99,7 @@ def lib() -> ctypes.CDLL:
         L.moin_route_workspace_bytes.argtypes = [i32, i32, i32]
         L.moin_route.argtypes = [ctypes.POINTER(_Router), vp, i32, vp, vp, vp, vp, sz, vp]
         L.moin_route_static.argtypes = [ctypes.POINTER(_Router), vp, i32, vp, vp, vp, vp]
+        L.moin_kmeans_update.argtypes = [ctypes.POINTER(_Plan), vp, vp, vp, vp, i32, vp]
         L.moin_plan_bytes.restype = sz
         L.moin_plan_bytes.argtypes = [i32, i32]
         L.moin_plan_build.argtypes = [vp, ctypes.POINTER(_Plan), vp]
@@ -225,6 +227,19 @@ def route_static(router: Router, queries: torch.Tensor, out_expert: torch.Tensor
     _check(lib().moin_route_static(ctypes.byref(router.c), _ptr(queries), queries.shape[0], _ptr(out_expert),
                                    _ptr(out_centroid), _ptr(out_best_sim), _stream(stream)), "moin_route_static")
     return out_expert
+
+
+def kmeans_update(plan: "Plan", x: torch.Tensor, centroids_old: torch.Tensor,
+                  centroids_new: Optional[torch.Tensor] = None, inv_norm_new: Optional[torch.Tensor] = None,
+                  stream=None) -> torch.Tensor:
+    """moin_kmeans_update: centroid k <- mean of the points the plan groups under cluster k."""
+    assert x.dtype == torch.bfloat16 and centroids_old.dtype == torch.bfloat16 and x.dim() == 2
+    assert centroids_old.shape == (plan.E, x.shape[1]) and plan.T == x.shape[0]
+    if centroids_new is None:
+        centroids_new = torch.empty_like(centroids_old)
+    _check(lib().moin_kmeans_update(ctypes.byref(plan.c), _ptr(x), _ptr(centroids_old), _ptr(centroids_new),
+                                    _ptr(inv_norm_new), x.shape[1], _stream(stream)), "moin_kmeans_update")
+    return centroids_new
 
 
 class Pool:

@@ -164,7 +164,7 @@ moin_status moin_profile_read(moin_profile_record* out, int32_t capacity, int32_
 const char* moin_kernel_name(int32_t k) {
   static const char* names[MOIN_K_COUNT] = {"route_simple", "route_tc", "route_finish", "plan", "gemm_warp", "gemm_tc",
                                             "lora_shrink_stream", "lora_expand_stream", "lora_shrink_tc",
-                                            "lora_fused_tc", "decoder_glue", "attention", "route_cluster"};
+                                            "lora_fused_tc", "decoder_glue", "attention", "route_cluster", "kmeans_update"};
   return (k >= 0 && k < MOIN_K_COUNT) ? names[k] : "unknown";
 }
 
@@ -279,6 +279,37 @@ moin_status moin_route_static(const moin_router* router, const void* queries, in
   ProfScope prof(MOIN_K_ROUTE_FINISH, 1, s);
   return record_cuda(launch_route_finish(keys, (const __nv_bfloat16*)queries, router->centroid_to_expert, Q, D,
                                          out_expert, out_centroid, out_best_sim, s));
+}
+
+/* ------------------------------------------------------------------ K-means update */
+
+moin_status moin_kmeans_update(const moin_plan* plan, const void* x, const void* centroids_old, void* centroids_new,
+                               float* inv_norm_new, int32_t D, moin_stream stream) {
+  if (!plan || plan->T < 0 || plan->E < 1 || !centroids_old || !centroids_new) return MOIN_ERR_INVALID_ARG;
+  if (D < 8 || D > 8192 || (D % 8) != 0) return MOIN_ERR_BAD_SHAPE;
+  if (plan->T > 0 && (!x || !plan->buffer)) return MOIN_ERR_INVALID_ARG;
+  if (!aligned16(centroids_old) || !aligned16(centroids_new) || (x && !aligned16(x))) return MOIN_ERR_MISALIGNED;
+  HostState* hs;
+  moin_status st = host_state(&hs);
+  if (st) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int K = plan->E;
+  if (centroids_new != centroids_old) {   // clusters without members keep their centroid
+    cudaError_t e = cudaMemcpyAsync(centroids_new, centroids_old, (size_t)K * (size_t)D * sizeof(__nv_bfloat16),
+                                    cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return record_cuda(e);
+  }
+  if (plan->T > 0) {
+    PlanView pv = plan_view(plan->buffer, plan->T, plan->E);
+    ProfScope prof(MOIN_K_KMEANS_UPDATE, 1, s);
+    st = record_cuda(launch_kmeans_mean(pv, (const __nv_bfloat16*)x, (__nv_bfloat16*)centroids_new, D, hs->n_sms, s));
+    if (st) return st;
+  }
+  if (inv_norm_new) {
+    ProfScope prof(MOIN_K_GLUE, 1, s);
+    return record_cuda(launch_inv_norm((const __nv_bfloat16*)centroids_new, K, D, inv_norm_new, s));
+  }
+  return MOIN_OK;
 }
 
 /* ------------------------------------------------------------------ plan */

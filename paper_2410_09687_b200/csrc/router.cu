@@ -344,6 +344,70 @@ cudaError_t launch_route_cluster(const __nv_bfloat16* q, const __nv_bfloat16* c,
   return cudaGetLastError();
 }
 
+// ----------------------------------------------------------------------------------------
+// K-means update: centroid of every non-empty cluster = mean of its member rows.  One CTA per segment of
+// the plan built from the assignments (segment = cluster id, start, length in `perm`, members in
+// increasing point order); thread c owns the 8 columns 8c..8c+7 and adds the member rows in order
+// (fp32), four rows' loads in flight at a time; the member indices are staged in shared memory 128 at a
+// time.  HBM-bound: every point is read once.
+// ----------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+kmeans_mean_kernel(const int* __restrict__ header, const int* __restrict__ perm, const int4* __restrict__ seg_tab,
+                   const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ c_new, int D) {
+  __shared__ int s_rows[128];
+  const int nseg = header[PH_NSEG];
+  const int tid = threadIdx.x, nch = D / 8;
+  for (int seg = blockIdx.x; seg < nseg; seg += gridDim.x) {
+    const int4 e = __ldg(seg_tab + seg);   // (cluster, start, length, -)
+    const int k = e.x, start = e.y, len = e.z;
+    for (int c0 = 0; c0 < nch; c0 += 128) {
+      const int ch = c0 + tid;
+      const bool on = ch < nch;
+      float acc[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+      for (int j0 = 0; j0 < len; j0 += 128) {
+        __syncthreads();
+        if (j0 + tid < len) s_rows[tid] = perm[start + j0 + tid];
+        __syncthreads();
+        const int nb = min(128, len - j0);
+        for (int j = 0; j < nb; j += 4) {
+          uint4 v[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            v[u] = (on && j + u < nb) ? ldg_stream(x + (size_t)s_rows[j + u] * D + ch * 8) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {   // rows added in member order; absent rows add zero
+            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              acc[2 * q] += bf16_lo(w[q]);
+              acc[2 * q + 1] += bf16_hi(w[q]);
+            }
+          }
+        }
+      }
+      if (on) {
+        const float n = (float)len;
+        uint4 o;
+        o.x = pack_bf16(acc[0] / n, acc[1] / n);
+        o.y = pack_bf16(acc[2] / n, acc[3] / n);
+        o.z = pack_bf16(acc[4] / n, acc[5] / n);
+        o.w = pack_bf16(acc[6] / n, acc[7] / n);
+        *reinterpret_cast<uint4*>(c_new + (size_t)k * D + ch * 8) = o;
+      }
+    }
+  }
+}
+
+cudaError_t launch_kmeans_mean(const PlanView& pv, const __nv_bfloat16* x, __nv_bfloat16* c_new, int D, int n_sms,
+                               cudaStream_t stream) {
+  long grid = pv.Smax < (long)n_sms * 16 ? pv.Smax : (long)n_sms * 16;
+  if (grid < 1) grid = 1;
+  kmeans_mean_kernel<<<(int)grid, 128, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, x, c_new, D);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_inv_norm(const __nv_bfloat16* c, int K, int D, float* inv_norm, cudaStream_t stream) {
   centroid_inv_norm_kernel<<<(K + 7) / 8, 256, 0, stream>>>(c, K, D, inv_norm);
   return cudaGetLastError();
