@@ -7,6 +7,8 @@ A "step" is one pass of the whole hot path over one batch of synthetic input:
   prefill: route 32 queries over 5 000 centroids -> plan -> seven projections, 32 x 512 tokens,
            5 000 rank-16 experts, Zipf(1.1) request experts
   router:  65 536 queries x 5 000 centroids x 768
+  kmeans:  one Lloyd iteration of the topic clustering: 65 536 points x 5 000 centroids x 768 (assign with the
+           router, group with the plan, update the centroids and their norms)
   forward: 22-block decoder, 64 x 256 tokens, 500 rank-64 experts on all seven projections
 
 `value` is device-timed throughput with inputs resident in HBM; `e2e` repeats the measurement
@@ -288,6 +290,62 @@ class RouterWorkload:
         return time.perf_counter() - t0
 
 
+class KMeansWorkload:
+    """One K-means (Lloyd) iteration over the router-stress data: assign, group, update (in place)."""
+
+    def __init__(self, dev: str, N: int = 65536, K: int = 5000, D: int = 768):
+        import paper_2410_09687_b200 as moin
+        self.moin, self.dev, self.N, self.K, self.D = moin, dev, N, K, D
+        rc = mi.planted_router(K, N, D, 3, device=dev)
+        g = torch.Generator(device=dev).manual_seed(7)
+        start = (rc.centroids.float() + 0.4 * torch.randn(K, D, generator=g, device=dev) / D ** 0.5).to(torch.bfloat16)
+        self.start = start
+        self.cent = start.clone()                  # updated in place every step
+        self.router = moin.Router(self.cent)       # borrows self.cent and owns the inverse norms
+        self.points = [rc.queries] + [torch.roll(rc.queries, shifts=i * 4099, dims=0).contiguous() for i in range(1, ROTATE)]
+        self.assign = torch.empty(N, dtype=torch.int32, device=dev)
+        self.plan = moin.Plan(N, K, dev, moin.PLAN_SEGMENTS)
+        self.router.workspace(N)
+        self.unit, self.units_per_step = "points", N
+        self.h_x = [self.points[0].cpu().pin_memory()]
+        self.h_c = torch.empty(K, D, dtype=torch.bfloat16).pin_memory()
+        self.d_x = torch.empty_like(rc.queries)
+        self.h2d, self.d2h = N * D * 2, K * D * 2
+
+    def _iterate(self, x):
+        moin = self.moin
+        moin.route(self.router, x, out_expert=self.assign)
+        moin.plan_build(self.assign, self.K, moin.PLAN_SEGMENTS, plan=self.plan)
+        moin.kmeans_update(self.plan, x, self.cent, centroids_new=self.cent, inv_norm_new=self.router.inv_norm)
+
+    def step(self, i: int):
+        self._iterate(self.points[i % ROTATE])
+
+    def step_e2e(self, i: int):
+        self.d_x.copy_(self.h_x[0], non_blocking=True)
+        self._iterate(self.d_x)
+        self.h_c.copy_(self.cent, non_blocking=True)
+
+    def config(self) -> dict:
+        return {"workload": f"k-means iteration: {self.N} points x {self.K} centroids x {self.D}, planted clusters, "
+                            f"perturbed start; assign (router) + group (plan) + update",
+                "l2": f"point matrix (100.7 MB) rotates over {ROTATE} buffers (> L2 in total)"}
+
+    def algorithmic(self) -> dict:
+        return {"flops": 2.0 * self.N * self.K * self.D,
+                "bytes": (self.N + 2 * self.K) * self.D * 2 + self.N * 4,
+                "update_bytes": (self.N + self.K) * self.D * 2 + self.N * 4}
+
+    def oracle_sample(self, n: int) -> float:
+        import oracle
+        x = mi.bf16_bits(self.points[0][:n])
+        c = mi.bf16_bits(self.start)
+        t0 = time.perf_counter()
+        a = oracle.route(x, c)["centroid"]
+        oracle.kmeans_update(x, c, a)
+        return time.perf_counter() - t0
+
+
 class ForwardWorkload:
     """22-block decoder, 64 x 256 tokens, 500 rank-64 experts on all 7 projections (pool ~50 GB)."""
 
@@ -479,14 +537,19 @@ def run_reference(args):
     oracle.build()
     cores = oracle.num_threads()
     kind = args.workload
-    rng_seed = {"decode": 1, "prefill": 2, "router": 3, "forward": 4}[kind]
-    if kind == "router":
+    rng_seed = {"decode": 1, "prefill": 2, "router": 3, "forward": 4, "kmeans": 3}[kind]
+    if kind in ("router", "kmeans"):
         n, K, D = 256, 5000, 768
         rc = mi.planted_router(K, n, D, rng_seed)
         q, c = mi.bf16_bits(rc.queries), mi.bf16_bits(rc.centroids)
-        fn = lambda: oracle.route(q, c)
-        unit, metric, sample = "queries/s", "router_queries_per_s", f"{n} of 65536 queries per step, all 5000 centroids"
-        cfgname = "router stress: 65536 queries x 5000 centroids x 768, planted clusters"
+        if kind == "router":
+            fn = lambda: oracle.route(q, c)
+            unit, metric, sample = "queries/s", "router_queries_per_s", f"{n} of 65536 queries per step, all 5000 centroids"
+            cfgname = "router stress: 65536 queries x 5000 centroids x 768, planted clusters"
+        else:
+            fn = lambda: oracle.kmeans_update(q, c, oracle.route(q, c)["centroid"])
+            unit, metric, sample = "points/s", "kmeans_points_per_s", f"assign + update of {n} of 65536 points per step, all 5000 centroids"
+            cfgname = "k-means iteration: 65536 points x 5000 centroids x 768, planted clusters"
     else:
         if kind == "forward":
             sys.stderr.write("[bench] reference arm for 'forward' times the seven projections of one block\n")
@@ -533,7 +596,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="moin", choices=["moin", "reference"])
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "router", "forward"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "router", "forward", "kmeans"])
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-router-extra", action="store_true")
@@ -542,7 +605,7 @@ def main():
     ap.add_argument("--rank", type=int, default=None, help="decode / prefill at another LoRA rank than the config's (side measurement)")
     ap.add_argument("--stream-impl", type=int, default=0, help="short-segment LoRA kernels: 0 auto, 1 register-fed, 2 TMA-staged")
     args = ap.parse_args()
-    defaults = {"decode": (3000, 20), "prefill": (100, 5), "router": (50, 5), "forward": (5, 3)}
+    defaults = {"decode": (3000, 20), "prefill": (100, 5), "router": (50, 5), "forward": (5, 3), "kmeans": (50, 5)}
     if args.impl == "reference":
         args.steps = args.steps if args.steps is not None else 5
         args.warmup = args.warmup if args.warmup is not None else 1
@@ -568,6 +631,8 @@ def main():
         wl = LayerWorkload(kind, dev, grouped=not args.no_group, rank=args.rank)
     elif kind == "router":
         wl = RouterWorkload(dev)
+    elif kind == "kmeans":
+        wl = KMeansWorkload(dev)
     else:
         wl = ForwardWorkload(dev, n_layers=args.forward_layers)
     torch.cuda.synchronize()
@@ -627,10 +692,16 @@ def main():
                     "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "frac_burst": ach / peaks["bf16_tflops"],
                     "frac_nominal": ach / NOMINAL_BF16_TFLOPS, "peak_source": peaks["source"] + " (sustained)",
                     "algorithmic_flops_per_launch": fl, "avg_launch_ms": sec * 1e3, "traffic": traffic_for(top, kind)}
-    elif kind == "router":
+    elif kind in ("router", "kmeans"):
         alg = wl.algorithmic()
         a = agg[top]
         sec = a["ms"] * 1e-3 / a["launches"]
+        if kind == "kmeans" and "kmeans_update" in agg:
+            u = agg["kmeans_update"]
+            usec = u["ms"] * 1e-3 / u["launches"]
+            extra["kmeans_update"] = {"bound": "hbm", "achieved": alg["update_bytes"] / usec / 1e9, "unit": "GB/s",
+                                      "peak": peaks["hbm_gbs"], "frac": alg["update_bytes"] / usec / 1e9 / peaks["hbm_gbs"],
+                                      "algorithmic_bytes_per_launch": alg["update_bytes"], "avg_launch_ms": usec * 1e3}
         ach = alg["flops"] / sec / 1e12
         tensor = top == "route_tc"
         roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
@@ -672,13 +743,17 @@ def main():
             n, t = adaptive_oracle(wl.oracle_sample, 64, 4096)
             cpu = {"value": n / t, "unit": "queries/s", "cores": oracle.num_threads(), "kind": "oracle",
                    "sample": f"{n} of {wl.Q} queries against all {wl.K} centroids, {t:.1f} s"}
+        elif kind == "kmeans":
+            n, t = adaptive_oracle(wl.oracle_sample, 64, 4096)
+            cpu = {"value": n / t, "unit": "points/s", "cores": oracle.num_threads(), "kind": "oracle",
+                   "sample": f"assign + update of {n} of {wl.N} points against all {wl.K} centroids, {t:.1f} s"}
         else:
             n, t = adaptive_oracle(wl.oracle_sample, 16, 256)
             cpu = {"value": n / t, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
                    "sample": f"route + 7 projections of the first {n} of {wl.T} tokens of one batch, {t:.1f} s"}
 
     if rank == 0:
-        metric = "router_queries_per_s" if kind == "router" else "routed_lora_tokens_per_s"
+        metric = {"router": "router_queries_per_s", "kmeans": "kmeans_points_per_s"}.get(kind, "routed_lora_tokens_per_s")
         cfg = wl.config()
         cfg.update({"launch": "cuda_graph replay of one step" if graphed else "plain stream launches",
                     "replicas": world, "peaks": peaks})

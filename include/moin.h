@@ -177,7 +177,9 @@ typedef struct {
  *   - a stable permutation of token indices ordered by expert id, with one segment
  *     (expert, start, length) per distinct expert - used when segments are short (decode);
  *   - the list of row tiles: maximal runs of consecutive tokens with one expert, cut into
- *     pieces of at most 128 rows - used when runs are long (prefill).
+ *     pieces of at most 128 rows - used when runs are long (prefill).  A build with mode
+ *     MOIN_PLAN_SEGMENTS leaves this list empty (nothing in that mode reads it): such a plan
+ *     must be rebuilt, not relabelled, before it is used as MOIN_PLAN_TILES.
  * Token expert ids: -1 = no expert (base model only); ids outside [-1, E) are treated as -1
  * and counted in moin_device_status.
  * ------------------------------------------------------------------------------------- */

@@ -333,7 +333,8 @@ moin_status moin_plan_build(const int32_t* token_expert, moin_plan* plan, moin_s
   PlanView v = plan_view(plan->buffer, plan->T, plan->E);
   {
     ProfScope prof(MOIN_K_PLAN, plan_launches(plan->T, plan->E), s);
-    st = record_cuda(launch_plan_build(token_expert, v, hs->status, s));
+    // the tile list serves the long-run kernels and the AUTO decision; a SEGMENTS plan leaves it empty
+    st = record_cuda(launch_plan_build(token_expert, v, hs->status, plan->mode != MOIN_PLAN_SEGMENTS, s));
   }
   if (st) return st;
   if (plan->mode == MOIN_PLAN_AUTO) {

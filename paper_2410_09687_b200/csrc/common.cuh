@@ -109,7 +109,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // Launchers implemented in the .cu files (host side).
 int plan_launches(int T, int E);   // kernels launch_plan_build issues for this shape
-cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, DeviceStatus* status, cudaStream_t stream);
+cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, DeviceStatus* status, bool want_tiles,
+                              cudaStream_t stream);
 // Register-fed short-segment kernels: one launch covers up to kMaxStreamJobs projections sharing a plan.
 constexpr int kMaxStreamJobs = 4;
 struct ShrinkJobs {

@@ -103,12 +103,13 @@ __global__ void __launch_bounds__(256) plan_prefix_kernel(PlanView v) {
   if (k > v.E) return;
   const size_t pitch = (size_t)(v.E + 1);
   int run = 0;
-  for (int c0 = 0; c0 < v.n_chunks; c0 += 8) {
-    int n[8];
+  constexpr int kBatch = 32;   // dependent round trips = chunks / kBatch
+  for (int c0 = 0; c0 < v.n_chunks; c0 += kBatch) {
+    int n[kBatch];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) n[j] = (c0 + j < v.n_chunks) ? __ldcg(v.hist + (size_t)(c0 + j) * pitch + k) : 0;
+    for (int j = 0; j < kBatch; ++j) n[j] = (c0 + j < v.n_chunks) ? __ldcg(v.hist + (size_t)(c0 + j) * pitch + k) : 0;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < kBatch; ++j) {
       if (c0 + j < v.n_chunks) v.hist[(size_t)(c0 + j) * pitch + k] = run;
       run += n[j];
     }
@@ -154,7 +155,7 @@ __device__ __forceinline__ void plan_tiles(const PlanView& v, const int* key, in
   for (int i = tid; i < carry_tiles; i += NT) v.tile_rows[i] = row0[i + 1] - row0[i];
 }
 
-__global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_prefix) {
+__global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_prefix, int want_tiles) {
   constexpr int NT = 1024;
   __shared__ int smem[33];
   __shared__ int s_carry[2];
@@ -206,8 +207,9 @@ __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_pref
     v.header[PH_E] = E;
   }
 
-  // 3. row tiles
-  plan_tiles<NT>(v, v.key, smem, s_carry, v.tile_row0);
+  // 3. row tiles (only the long-run kernels read them)
+  if (want_tiles) plan_tiles<NT>(v, v.key, smem, s_carry, v.tile_row0);
+  else if (tid == 0) v.header[PH_NTILES] = 0;
 }
 
 // Whole plan of a batch of at most 1024 tokens in one CTA.  The tokens are sorted by the key
@@ -218,7 +220,7 @@ constexpr int kPlanSmallT = 1024;
 constexpr int kPlanSmallE = 1 << 20;   // the id must fit above the 10 token bits of a 31-bit key
 template <int NT>   // threads = sort width: the power of two at or above T, at least 128
 __global__ void __launch_bounds__(NT) plan_small_kernel(const int* __restrict__ token_expert, PlanView v,
-                                                        DeviceStatus* status) {
+                                                        DeviceStatus* status, int want_tiles) {
   __shared__ int s_key[NT];        // sanitised id by token
   __shared__ int s_sort[NT];       // sort keys, then the segment starts
   __shared__ int s_row0[NT + 1];   // tile starts
@@ -282,7 +284,8 @@ __global__ void __launch_bounds__(NT) plan_small_kernel(const int* __restrict__ 
     v.header[PH_T] = T;
     v.header[PH_E] = E;
   }
-  plan_tiles<NT>(v, s_key, smem, s_carry, s_row0);
+  if (want_tiles) plan_tiles<NT>(v, s_key, smem, s_carry, s_row0);
+  else if (tid == 0) v.header[PH_NTILES] = 0;
 }
 
 __global__ void __launch_bounds__(kPlanChunk) plan_scatter_kernel(PlanView v) {
@@ -298,19 +301,20 @@ int plan_launches(int T, int E) {
   return T > kPlanChunk ? 4 : 3;
 }
 
-cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, DeviceStatus* status, cudaStream_t stream) {
+cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, DeviceStatus* status, bool want_tiles,
+                              cudaStream_t stream) {
   if (v.T <= kPlanSmallT && v.E < kPlanSmallE) {
-    if (v.T <= 128) plan_small_kernel<128><<<1, 128, 0, stream>>>(token_expert, v, status);
-    else if (v.T <= 256) plan_small_kernel<256><<<1, 256, 0, stream>>>(token_expert, v, status);
-    else if (v.T <= 512) plan_small_kernel<512><<<1, 512, 0, stream>>>(token_expert, v, status);
-    else plan_small_kernel<1024><<<1, 1024, 0, stream>>>(token_expert, v, status);
+    if (v.T <= 128) plan_small_kernel<128><<<1, 128, 0, stream>>>(token_expert, v, status, want_tiles);
+    else if (v.T <= 256) plan_small_kernel<256><<<1, 256, 0, stream>>>(token_expert, v, status, want_tiles);
+    else if (v.T <= 512) plan_small_kernel<512><<<1, 512, 0, stream>>>(token_expert, v, status, want_tiles);
+    else plan_small_kernel<1024><<<1, 1024, 0, stream>>>(token_expert, v, status, want_tiles);
     return cudaGetLastError();
   }
   cudaError_t e = cudaMemsetAsync(v.hist, 0, sizeof(int) * (size_t)v.n_chunks * (size_t)(v.E + 1), stream);
   if (e != cudaSuccess) return e;
   plan_rank_kernel<<<v.n_chunks, kPlanChunk, 0, stream>>>(token_expert, v.T, v.E, v.key, v.rank, v.hist, status);
   if (v.n_chunks > 1) plan_prefix_kernel<<<(v.E + 1 + 255) / 256, 256, 0, stream>>>(v);
-  plan_scan_kernel<<<1, 1024, 0, stream>>>(v, v.n_chunks > 1 ? 0 : 1);
+  plan_scan_kernel<<<1, 1024, 0, stream>>>(v, v.n_chunks > 1 ? 0 : 1, want_tiles);
   plan_scatter_kernel<<<v.n_chunks, kPlanChunk, 0, stream>>>(v);
   return cudaGetLastError();
 }
