@@ -169,6 +169,41 @@ typedef struct {
 } moin_pool;
 
 /* ---------------------------------------------------------------------------------------
+ * Two-tier adapter store.  Paper Sec. 1: the adapters are small enough to be stored in bulk and the ones in
+ * use are kept in GPU memory; fetching a missing one costs latency.  Here every expert's adapters stay in
+ * HOST memory (E stacked adapters per projection, same layout as a pool), the device pools hold n_slots of
+ * them, and moin_cache_admit - called between the router and the forward pass with the batch's expert ids on
+ * the host - makes every expert of the batch resident: a hit only refreshes its age, a miss takes a free slot
+ * or else the least recently used slot that this batch does not need, and enqueues one host-to-device copy
+ * per matrix and projection on `stream`.  It then uploads the expert -> slot table (-1 = not resident) that
+ * all the pools of the store share as their slot_of_expert.  Kernels already enqueued on `stream` still see
+ * the old contents; everything enqueued after the call sees the batch's experts in place.
+ *
+ *   host_A [E, r, d_in], host_B [E, d_out, r]   host bf16, pinned for truly asynchronous copies
+ *   dev_A [n_slots, r, d_in], dev_B [n_slots, d_out, r]   device bf16: the A / B of the projection's moin_pool
+ * The object is host state plus a few small pinned staging buffers; it allocates no device memory.  One
+ * thread at a time.  Errors: INVALID_ARG; WORKSPACE when a batch names more distinct experts than there are
+ * slots (nothing is copied then); ids outside [0, E) are skipped (they mean "no adapter").
+ * ------------------------------------------------------------------------------------- */
+typedef struct moin_cache moin_cache;
+typedef struct {
+  const void* host_A;
+  const void* host_B;
+  void* dev_A;
+  void* dev_B;
+  int32_t r, d_in, d_out;
+} moin_cache_projection;
+moin_status moin_cache_create(int32_t E, int32_t n_slots, const moin_cache_projection* projs, int32_t n_projs,
+                              int32_t* dev_slot_of_expert /* [E] device */, moin_cache** out);
+void moin_cache_destroy(moin_cache* cache);
+/* expert_ids: HOST array of n ids (one per request or token, repeats allowed).  n_missed / bytes_copied
+ * (nullable): experts brought in by this call and the bytes of their copies. */
+moin_status moin_cache_admit(moin_cache* cache, const int32_t* expert_ids, int32_t n, moin_stream stream,
+                             int32_t* n_missed, uint64_t* bytes_copied);
+/* Slot an expert occupies after the last admit (-1 = not resident); host bookkeeping only. */
+moin_status moin_cache_slot_of(const moin_cache* cache, int32_t expert, int32_t* slot);
+
+/* ---------------------------------------------------------------------------------------
  * Batch plan = the grouping of a batch's tokens by expert.  Paper Sec. 1 names the need
  * (many adapters in one batch) and Sec. 3.3 fixes that the expert is per request, so the
  * plan is built once per batch and reused by every projection of every block.

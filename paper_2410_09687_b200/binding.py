@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = (
     "moin_plan_build", "moin_plan_read", "moin_lora_linear_workspace_bytes", "moin_lora_linear",
     "moin_decoder_workspace_bytes", "moin_decoder_forward", "moin_profile_enable", "moin_profile_read",
     "moin_kernel_name", "moin_route_static", "moin_lora_linear_group", "moin_lora_linear_group_workspace_bytes",
-    "moin_kmeans_update",
+    "moin_kmeans_update", "moin_cache_create", "moin_cache_destroy", "moin_cache_admit", "moin_cache_slot_of",
 )
 
 
@@ -44,6 +44,11 @@ class _Pool(ctypes.Structure):
 
 class _Job(ctypes.Structure):
     _fields_ = [("x", ctypes.c_void_p), ("W", ctypes.c_void_p), ("pool", ctypes.POINTER(_Pool)), ("y", ctypes.c_void_p)]
+
+
+class _CacheProj(ctypes.Structure):
+    _fields_ = [("host_A", ctypes.c_void_p), ("host_B", ctypes.c_void_p), ("dev_A", ctypes.c_void_p),
+                ("dev_B", ctypes.c_void_p), ("r", ctypes.c_int32), ("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32)]
 
 
 class _Plan(ctypes.Structure):
@@ -100,6 +105,11 @@ def lib() -> ctypes.CDLL:
         L.moin_route.argtypes = [ctypes.POINTER(_Router), vp, i32, vp, vp, vp, vp, sz, vp]
         L.moin_route_static.argtypes = [ctypes.POINTER(_Router), vp, i32, vp, vp, vp, vp]
         L.moin_kmeans_update.argtypes = [ctypes.POINTER(_Plan), vp, vp, vp, vp, i32, vp]
+        L.moin_cache_create.argtypes = [i32, i32, ctypes.POINTER(_CacheProj), i32, vp, ctypes.POINTER(vp)]
+        L.moin_cache_destroy.restype = None
+        L.moin_cache_destroy.argtypes = [vp]
+        L.moin_cache_admit.argtypes = [vp, vp, i32, vp, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_uint64)]
+        L.moin_cache_slot_of.argtypes = [vp, i32, ctypes.POINTER(i32)]
         L.moin_plan_bytes.restype = sz
         L.moin_plan_bytes.argtypes = [i32, i32]
         L.moin_plan_build.argtypes = [vp, ctypes.POINTER(_Plan), vp]
@@ -227,6 +237,58 @@ def route_static(router: Router, queries: torch.Tensor, out_expert: torch.Tensor
     _check(lib().moin_route_static(ctypes.byref(router.c), _ptr(queries), queries.shape[0], _ptr(out_expert),
                                    _ptr(out_centroid), _ptr(out_best_sim), _stream(stream)), "moin_route_static")
     return out_expert
+
+
+class AdapterCache:
+    """moin_cache: all experts' adapters in host memory, ``n_slots`` of them resident in the device pools.
+
+    ``host`` is a list of (A [E, r, d_in], B [E, d_out, r]) CPU bf16 tensors (pinned for asynchronous copies), one
+    pair per projection.  The device pools (``self.pools``) share one expert -> slot table."""
+
+    def __init__(self, host: Sequence[tuple], n_slots: int, device):
+        self.host = [(A, B) for A, B in host]
+        E = self.host[0][0].shape[0]
+        self.E, self.n_slots = E, n_slots
+        self.table = torch.full((E,), -1, dtype=torch.int32, device=device)
+        self.pools, descs = [], (_CacheProj * len(self.host))()
+        for i, (A, B) in enumerate(self.host):
+            assert A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16 and not A.is_cuda and not B.is_cuda
+            assert A.is_contiguous() and B.is_contiguous() and A.shape[0] == E and B.shape[0] == E
+            _, r, d_in = A.shape
+            d_out = B.shape[1]
+            dA = torch.zeros(n_slots, r, d_in, dtype=torch.bfloat16, device=device)
+            dB = torch.zeros(n_slots, d_out, r, dtype=torch.bfloat16, device=device)
+            self.pools.append(Pool(dA, dB, self.table))
+            descs[i] = _CacheProj(A.data_ptr(), B.data_ptr(), dA.data_ptr(), dB.data_ptr(), r, d_in, d_out)
+        h = ctypes.c_void_p()
+        _check(lib().moin_cache_create(E, n_slots, descs, len(self.host), _ptr(self.table), ctypes.byref(h)),
+               "moin_cache_create")
+        self.handle = h
+
+    def admit(self, expert_ids, stream=None) -> dict:
+        """moin_cache_admit with the batch's expert ids (host int32 array-like).  Returns misses and bytes copied."""
+        import numpy as _np
+        ids = _np.ascontiguousarray(expert_ids, dtype=_np.int32)
+        missed, nbytes = ctypes.c_int32(0), ctypes.c_uint64(0)
+        _check(lib().moin_cache_admit(self.handle, ids.ctypes.data, ids.shape[0], _stream(stream), ctypes.byref(missed),
+                                      ctypes.byref(nbytes)), "moin_cache_admit")
+        return {"missed": missed.value, "bytes": nbytes.value}
+
+    def slot_of(self, expert: int) -> int:
+        s = ctypes.c_int32(0)
+        _check(lib().moin_cache_slot_of(self.handle, expert, ctypes.byref(s)), "moin_cache_slot_of")
+        return s.value
+
+    def close(self):
+        if self.handle is not None:
+            lib().moin_cache_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def kmeans_update(plan: "Plan", x: torch.Tensor, centroids_old: torch.Tensor,
