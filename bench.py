@@ -110,7 +110,7 @@ class ClockSampler:
 class LayerWorkload:
     """route -> plan -> seven projections.  decode: E=500 r=64 T=256; prefill: E=5000 r=16 32x512."""
 
-    def __init__(self, kind: str, dev: str, grouped: bool = True, rank=None):
+    def __init__(self, kind: str, dev: str, grouped: bool = True, rank=None, cache_slots=None):
         import paper_2410_09687_b200 as moin
         self.moin, self.kind, self.dev, self.grouped = moin, kind, dev, grouped
         if kind == "decode":
@@ -140,9 +140,21 @@ class LayerWorkload:
         else:
             self.routers = [self.router] * ROTATE
         self.pools, self.W, self.x, self.y = [], [], [], []
+        self.cache = None
+        if cache_slots:   # two-tier store: every expert's adapters in pinned host memory, cache_slots of them in HBM
+            host = []
+            for p, (name, d_in, d_out) in enumerate(self.projs):
+                pool = mi.make_pool(self.E, self.r, d_in, d_out, self.seed, 30 + p)
+                host.append((pool.A.contiguous().pin_memory(), pool.B.contiguous().pin_memory()))
+            self.cache = moin.AdapterCache(host, int(cache_slots), dev)
+            self.h_ids = torch.empty(self.R, dtype=torch.int32).pin_memory()
+            self.cache_misses, self.cache_bytes, self.cache_steps = 0, 0, 0
         for p, (name, d_in, d_out) in enumerate(self.projs):
-            pool = mi.make_pool(self.E, self.r, d_in, d_out, self.seed, 30 + p, device=dev)
-            self.pools.append(moin.Pool(pool.A, pool.B, pool.slot_of_expert))
+            if self.cache is not None:
+                self.pools.append(self.cache.pools[p])
+            else:
+                pool = mi.make_pool(self.E, self.r, d_in, d_out, self.seed, 30 + p, device=dev)
+                self.pools.append(moin.Pool(pool.A, pool.B, pool.slot_of_expert))
             self.W.append(mi.normal_bf16((d_out, d_in), 0.02, self.seed, 40 + p, 12, device=dev))
             self.x.append([mi.normal_bf16((self.T, d_in), 1.0, self.seed, 40 + p, 11, i, device=dev)
                            for i in range(ROTATE)])
@@ -173,6 +185,11 @@ class LayerWorkload:
     def _core(self, i: int, q, xs, jobgroups=None):
         moin = self.moin
         moin.route(self.routers[i], q, out_expert=self.req_expert)
+        if self.cache is not None:   # the router's ids go to the host, the batch's missing adapters come in
+            self.h_ids.copy_(self.req_expert, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            got = self.cache.admit(self.h_ids.numpy())
+            self.cache_misses += got["missed"]; self.cache_bytes += got["bytes"]; self.cache_steps += 1
         if self.kind == "decode":
             te = self.req_expert
         else:
@@ -602,6 +619,9 @@ def main():
     ap.add_argument("--no-router-extra", action="store_true")
     ap.add_argument("--forward-layers", type=int, default=22)
     ap.add_argument("--no-group", action="store_true", help="one moin_lora_linear call per projection")
+    ap.add_argument("--cache-slots", type=int, default=None,
+                    help="decode / prefill through the two-tier adapter store with this many device slots (side "
+                         "measurement: the step then contains a host round trip and the copies of the missing adapters)")
     ap.add_argument("--rank", type=int, default=None, help="decode / prefill at another LoRA rank than the config's (side measurement)")
     ap.add_argument("--stream-impl", type=int, default=0, help="short-segment LoRA kernels: 0 auto, 1 register-fed, 2 TMA-staged")
     args = ap.parse_args()
@@ -628,7 +648,7 @@ def main():
     peaks = load_peaks()
     kind = args.workload
     if kind in ("decode", "prefill"):
-        wl = LayerWorkload(kind, dev, grouped=not args.no_group, rank=args.rank)
+        wl = LayerWorkload(kind, dev, grouped=not args.no_group, rank=args.rank, cache_slots=args.cache_slots)
     elif kind == "router":
         wl = RouterWorkload(dev)
     elif kind == "kmeans":
@@ -636,7 +656,7 @@ def main():
     else:
         wl = ForwardWorkload(dev, n_layers=args.forward_layers)
     torch.cuda.synchronize()
-    use_graph = (not args.no_graph) and kind != "forward"
+    use_graph = (not args.no_graph) and kind != "forward" and not getattr(args, "cache_slots", None)
 
     sampler = ClockSampler(local)
     sampler.start()
@@ -661,6 +681,10 @@ def main():
     prof_steps = min(args.steps, 20)
     roof = None
     extra = {}
+    if kind in ("decode", "prefill") and wl.cache is not None and wl.cache_steps:
+        extra["adapter_cache"] = {"slots": wl.cache.n_slots, "experts": wl.E,
+                                  "misses_per_step": wl.cache_misses / wl.cache_steps,
+                                  "h2d_adapter_bytes_per_step": wl.cache_bytes / wl.cache_steps}
     if kind in ("decode", "prefill"):
         nd = wl.distinct()
         alg = wl.algorithmic(nd)
