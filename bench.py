@@ -244,13 +244,23 @@ class LayerWorkload:
                 "l2": f"inputs rotate over {ROTATE} batches; per-step working set exceeds L2"}
 
     def oracle_sample(self, n_tokens: int) -> float:
-        """Seconds the CPU oracle needs for route + the seven projections of the first n_tokens tokens of batch 0."""
+        """Seconds the CPU oracle needs for route + the seven projections of n_tokens tokens: the first tokens of
+        batch 0, then of batch 1, ... (a sample larger than one batch goes round the rotating batches)."""
         import oracle
+        total, done, b = 0.0, 0, 0
+        while done < n_tokens:
+            n = min(self.T, n_tokens - done)
+            total += self._oracle_batch(oracle, b % ROTATE, n)
+            done += n
+            b += 1
+        return total
+
+    def _oracle_batch(self, oracle, b: int, n_tokens: int) -> float:
         n_req = max(1, n_tokens * self.R // self.T)
         rows = np.arange(n_tokens)
-        q = mi.bf16_bits(self.queries[0][:n_req])
+        q = mi.bf16_bits(self.queries[b][:n_req])
         c = mi.bf16_bits(self.router.centroids)
-        self.step(0)
+        self.step(b)
         torch.cuda.synchronize()
         te = (self.req_expert if self.kind == "decode" else self.token_expert).cpu().numpy()[rows]
         used = sorted(set(int(e) for e in te if e >= 0))
@@ -259,7 +269,7 @@ class LayerWorkload:
         idx = torch.tensor(used, dtype=torch.long, device=self.dev)
         host = []
         for p, (_, d_in, d_out) in enumerate(self.projs):
-            host.append((mi.bf16_bits(self.x[p][0][:n_tokens]), mi.bf16_bits(self.W[p]),
+            host.append((mi.bf16_bits(self.x[p][b][:n_tokens]), mi.bf16_bits(self.W[p]),
                          mi.bf16_bits(self.pools[p].A[idx]), mi.bf16_bits(self.pools[p].B[idx])))
         t0 = time.perf_counter()
         oracle.route(q, c)
@@ -534,8 +544,9 @@ def traffic_for(kernel: str, workload: str):
         return None
 
 
-def adaptive_oracle(sample_fn, first: int, cap: int, target_s: float = 12.0):
-    """Times the oracle on `first` units, then once more on a sample sized for ~target_s seconds."""
+def adaptive_oracle(sample_fn, first: int, cap: int, target_s: float = 20.0):
+    """Times the oracle on `first` units, then once more on a sample sized from that rate for target_s seconds
+    (small samples run slower per unit, so the second run ends up around half of target_s)."""
     t = sample_fn(first)
     n = int(min(cap, max(first, first * target_s / max(t, 1e-3))))
     if n > first * 1.5:
@@ -772,9 +783,9 @@ def main():
             cpu = {"value": n / t, "unit": "points/s", "cores": oracle.num_threads(), "kind": "oracle",
                    "sample": f"assign + update of {n} of {wl.N} points against all {wl.K} centroids, {t:.1f} s"}
         else:
-            n, t = adaptive_oracle(wl.oracle_sample, 16, 256)
+            n, t = adaptive_oracle(wl.oracle_sample, 16, 16 * wl.T if kind == "decode" else 4096)
             cpu = {"value": n / t, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
-                   "sample": f"route + 7 projections of the first {n} of {wl.T} tokens of one batch, {t:.1f} s"}
+                   "sample": f"route + 7 projections of {n} tokens (batches of at most {wl.T}, step size {wl.T}), {t:.1f} s"}
 
     if rank == 0:
         metric = {"router": "router_queries_per_s", "kmeans": "kmeans_points_per_s"}.get(kind, "routed_lora_tokens_per_s")
