@@ -138,7 +138,7 @@ __device__ __forceinline__ void ldmatrix_x4_plain(uint32_t addr, uint32_t& r0, u
 __global__ void __launch_bounds__(128)
 attention_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                  const __nv_bfloat16* __restrict__ v, const int* __restrict__ cu, __nv_bfloat16* __restrict__ out,
-                 int n_heads, int n_kv_heads, float scale_log2) {
+                 int n_heads, int n_kv_heads, float scale_log2, const float2* __restrict__ rope) {
   __shared__ __align__(16) uint16_t Ks[2][64 * kAttPitch];
   __shared__ __align__(16) uint16_t Vs[2][64 * kAttPitch];
   const int req = blockIdx.z, head = blockIdx.y, qb = blockIdx.x;
@@ -177,6 +177,25 @@ attention_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
     qa[ks][1] = (r1 < L) ? *reinterpret_cast<const uint32_t*>(p1) : 0u;
     qa[ks][2] = (r0 < L) ? *reinterpret_cast<const uint32_t*>(p0 + 8) : 0u;
     qa[ks][3] = (r1 < L) ? *reinterpret_cast<const uint32_t*>(p1 + 8) : 0u;
+  }
+  if (rope != nullptr) {
+    // rotary embedding of the query rows on the fly (pairing (d, d + 32): k-steps ks and ks + 2 of the same
+    // thread; position = row index inside the request), rounded to bf16 as the stand-alone kernel does
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+      for (int idx = 0; idx < 4; ++idx) {
+        const int row = (idx & 1) ? r1 : r0;
+        if (row < L) {
+          const int d0 = ks * 16 + 2 * t + ((idx & 2) ? 8 : 0);
+          const float4 cc = __ldg(reinterpret_cast<const float4*>(rope + (size_t)row * 32 + d0));   // d0 is even
+          const float2 c0 = make_float2(cc.x, cc.y), c1 = make_float2(cc.z, cc.w);
+          const uint32_t lo = qa[ks][idx], hi = qa[ks + 2][idx];
+          const float a0 = bf16_lo(lo), a1 = bf16_hi(lo), b0 = bf16_lo(hi), b1 = bf16_hi(hi);
+          qa[ks][idx] = pack_bf16(a0 * c0.x - b0 * c0.y, a1 * c1.x - b1 * c1.y);
+          qa[ks + 2][idx] = pack_bf16(b0 * c0.x + a0 * c0.y, b1 * c1.x + a1 * c1.y);
+        }
+      }
   }
   float o[8][4];
 #pragma unroll
@@ -397,11 +416,13 @@ extern "C" moin_status moin_decoder_forward(const moin_model* m, const int32_t* 
       void* const outs[3] = {w.q, w.k, w.v};
       if ((st = proj_group(l, 0, 3, w.xn, din, dout, outs))) return st;
     }
-    { ProfScope prof(MOIN_K_GLUE, 2, s);
-      rope_kernel<<<(int)(((long)T * nh * 32 + 255) / 256), 256, 0, s>>>(w.q, w.pos, w.rope, T, nh);
+    // rotary embedding: the keys are rotated in place once (every query head and every later query reads them);
+    // the queries are rotated inside the attention kernel as it loads them
+    { ProfScope prof(MOIN_K_GLUE, 1, s);
       rope_kernel<<<(int)(((long)T * nkv * 32 + 255) / 256), 256, 0, s>>>(w.k, w.pos, w.rope, T, nkv); }
     { ProfScope prof(MOIN_K_ATTENTION, 1, s);
-      attention_kernel<<<dim3((max_seqlen + 63) / 64, nh, R), 128, 0, s>>>(w.q, w.k, w.v, cu_seqlens, w.att, nh, nkv, scale_log2); }
+      attention_kernel<<<dim3((max_seqlen + 63) / 64, nh, R), 128, 0, s>>>(w.q, w.k, w.v, cu_seqlens, w.att, nh, nkv, scale_log2,
+                                                                         w.rope); }
     if ((st = proj(l, 3, w.att, qd, H, w.o))) return st;
     { ProfScope prof(MOIN_K_GLUE, 1, s);
       add_rmsnorm_kernel<<<T, 256, 0, s>>>(w.res, w.o, (const __nv_bfloat16*)m->mlp_norm[l], w.xn, H, m->rms_eps, nullptr); }
