@@ -428,9 +428,24 @@ cudaError_t launch_route_simple(const __nv_bfloat16* q, const __nv_bfloat16* c, 
   return cudaGetLastError();
 }
 
+// The same without the cosine output: nothing to reduce, so one thread per query (coalesced keys and ids).
+__global__ void __launch_bounds__(256)
+route_finish_ids_kernel(const unsigned long long* __restrict__ keys, const int* __restrict__ cmap, int Q,
+                        int* __restrict__ out_expert, int* __restrict__ out_centroid) {
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= Q) return;
+  const unsigned long long key = keys[i];
+  const int id = (key == 0ull) ? 0 : (int)(0xFFFFFFFFu - (uint32_t)(key & 0xFFFFFFFFull));
+  if (out_centroid) out_centroid[i] = id;
+  out_expert[i] = cmap ? cmap[id] : id;
+}
+
 cudaError_t launch_route_finish(const unsigned long long* keys, const __nv_bfloat16* q, const int* cmap, int Q, int D,
                                 int* out_expert, int* out_centroid, float* out_best, cudaStream_t stream) {
-  route_finish_kernel<<<(Q + 7) / 8, 256, 0, stream>>>(keys, q, cmap, Q, D, out_expert, out_centroid, out_best);
+  if (out_best == nullptr)
+    route_finish_ids_kernel<<<(Q + 255) / 256, 256, 0, stream>>>(keys, cmap, Q, out_expert, out_centroid);
+  else
+    route_finish_kernel<<<(Q + 7) / 8, 256, 0, stream>>>(keys, q, cmap, Q, D, out_expert, out_centroid, out_best);
   return cudaGetLastError();
 }
 
