@@ -171,6 +171,32 @@ def test_grouped_projections_equal_single_calls(mode, stream_impl):
         assert_layer_close(y, oracle_layer(case), case.name)
 
 
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_seeded_random_shapes_in_every_plan_mode(seed):
+    # ranks, widths (also not multiples of 16 / 64), segment structures (runs, interleaved tokens, base-only
+    # tokens, out-of-range ids, experts without adapters) drawn at random; every mode against the oracle
+    rng = np.random.default_rng(seed)
+    for it in range(10):
+        r = int(rng.choice([8, 16, 24, 40, 64, 72, 128]))
+        d_in = int(rng.choice([64, 128, 192, 256, 320, 512, 1024, 2048]))
+        d_out = int(rng.choice([8, 24, 64, 72, 136, 256, 328, 512, 1000, 2048]))
+        E = int(rng.integers(1, 40))
+        n_req = int(rng.integers(1, 24))
+        lens = rng.integers(1, int(rng.choice([1, 3, 9, 40, 200])) + 1, size=n_req)
+        te = np.repeat(rng.integers(-1, E, size=n_req), lens).astype(np.int32)
+        if rng.random() < 0.3:
+            te = rng.permutation(te)
+        if rng.random() < 0.2:
+            te[rng.integers(0, len(te))] = E + 5
+        missing = tuple(int(m) for m in rng.choice(E, size=min(E - 1, int(rng.integers(0, 3))), replace=False)) if E > 1 else ()
+        pool = mi.make_pool(E, r, d_in, d_out, 100 * seed + it, 1, missing=missing)
+        case = mi.layer_case("random", len(te), d_in, d_out, pool, te, float(rng.choice([1.0, 2.0, 0.5])), 100 * seed + it, 2)
+        ref = oracle_layer(case)
+        for mode in (moin.PLAN_SEGMENTS, moin.PLAN_TILES, moin.PLAN_AUTO):
+            y, _ = run_layer(case, mode)
+            assert_layer_close(y, ref, f"seed {seed} case {it} mode {mode}: r {r}, {d_in}->{d_out}, E {E}, T {len(te)}")
+
+
 def test_empty_batch_and_argument_errors():
     pool = gpu_pool(mi.make_pool(4, 8, 64, 64, 10, 1))
     x = torch.zeros(0, 64, dtype=torch.bfloat16, device=DEV)
