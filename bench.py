@@ -841,6 +841,12 @@ def main():
             cpu = {"value": n / t, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
                    "sample": f"route + 7 projections of {n} tokens (batches of at most {wl.T}, step size {wl.T}), {t:.1f} s"}
 
+    if rank == 0 and kind in ("router", "decode", "prefill"):
+        # queries of the first batch whose two best cosines are closer than 1e-4 (reported by the library itself)
+        rq = wl.queries[0]
+        m = moin.route_top2(wl.router, rq)["margin"]
+        extra["near_ties"] = {"margin_below": 1e-4, "count": int((m < 1e-4).sum().item()), "of": int(rq.shape[0]),
+                              "min_margin": float(m.min().item())}
     if rank == 0:
         metric = {"router": "router_queries_per_s", "kmeans": "kmeans_points_per_s"}.get(kind, "routed_lora_tokens_per_s")
         cfg = wl.config()

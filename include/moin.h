@@ -130,6 +130,18 @@ moin_status moin_route(const moin_router* router, const void* queries, int32_t Q
                        int32_t* out_centroid, float* out_best_sim, void* workspace, size_t workspace_bytes,
                        moin_stream stream);
 
+/* Router with runner-up.  Paper Sec. 3.3 routes by nearest topic embedding; how far the nearest is ahead of the
+ * second nearest tells how safe that choice was (a query whose two best cosines differ by less than ~1e-4 sits
+ * between two topics: a different rounding order may route it to the other one).  Same arguments and rules as
+ * moin_route, plus
+ *   out_second  [Q] int32, nullable: centroid index of the second-best similarity, -1 if there is none
+ *   out_margin  [Q] fp32,  nullable: cos(best) - cos(second), +inf if there is no second candidate
+ * out_expert and out_centroid may be NULL here.  Workspace: moin_route_top2_workspace_bytes. */
+size_t moin_route_top2_workspace_bytes(int32_t Q, int32_t K, int32_t D);
+moin_status moin_route_top2(const moin_router* router, const void* queries, int32_t Q, int32_t* out_expert,
+                            int32_t* out_centroid, int32_t* out_second, float* out_best_sim, float* out_margin,
+                            void* workspace, size_t workspace_bytes, moin_stream stream);
+
 /* Routing for callers that cannot hand the library a workspace.  (The paper has no counterpart: this is
  * a packaging variant of moin_route, added for processes that must not allocate device memory - e.g. a
  * serving worker whose memory pool was sized and frozen at start-up, or a plug-in that runs inside

@@ -4,11 +4,11 @@ The binding only marshals arguments (torch tensors -> device pointers); every st
 path runs in the library's CUDA kernels.  There is no CPU or PyTorch fallback: if the
 library is missing or no sm_100 GPU is present, calls raise.
 """
-from .binding import (MoinError, Router, Pool, Plan, DecoderModel, lib, lib_path, route, route_static, ROUTE_STATIC_MAX_Q, plan_build, kmeans_update, AdapterCache, lora_linear, lora_linear_group, JobGroup,
+from .binding import (MoinError, Router, Pool, Plan, DecoderModel, lib, lib_path, route, route_top2, route_static, ROUTE_STATIC_MAX_Q, plan_build, kmeans_update, AdapterCache, lora_linear, lora_linear_group, JobGroup,
                       decoder_forward, device_status, device_status_reset, set_option, profile_enable, profile_read, PLAN_AUTO, PLAN_SEGMENTS,
                       PLAN_TILES, LOGITS_ALL, LOGITS_LAST, LOGITS_NONE, OPT_GEMM_IMPL, OPT_STREAM_IMPL, EXPORTED_SYMBOLS)
 
-__all__ = ["MoinError", "Router", "Pool", "Plan", "DecoderModel", "lib", "lib_path", "route", "route_static", "ROUTE_STATIC_MAX_Q", "plan_build", "kmeans_update", "AdapterCache",
+__all__ = ["MoinError", "Router", "Pool", "Plan", "DecoderModel", "lib", "lib_path", "route", "route_top2", "route_static", "ROUTE_STATIC_MAX_Q", "plan_build", "kmeans_update", "AdapterCache",
            "lora_linear", "lora_linear_group", "JobGroup", "decoder_forward", "device_status", "device_status_reset", "set_option", "profile_enable", "profile_read", "PLAN_AUTO",
            "PLAN_SEGMENTS", "PLAN_TILES", "LOGITS_ALL", "LOGITS_LAST", "LOGITS_NONE", "OPT_GEMM_IMPL", "OPT_STREAM_IMPL",
            "EXPORTED_SYMBOLS"]

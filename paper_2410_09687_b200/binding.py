@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = (
     "moin_plan_build", "moin_plan_read", "moin_lora_linear_workspace_bytes", "moin_lora_linear",
     "moin_decoder_workspace_bytes", "moin_decoder_forward", "moin_profile_enable", "moin_profile_read",
     "moin_kernel_name", "moin_route_static", "moin_lora_linear_group", "moin_lora_linear_group_workspace_bytes",
-    "moin_kmeans_update", "moin_cache_create", "moin_cache_destroy", "moin_cache_admit", "moin_cache_slot_of",
+    "moin_kmeans_update", "moin_route_top2", "moin_route_top2_workspace_bytes", "moin_cache_create", "moin_cache_destroy", "moin_cache_admit", "moin_cache_slot_of",
 )
 
 
@@ -105,6 +105,9 @@ def lib() -> ctypes.CDLL:
         L.moin_route.argtypes = [ctypes.POINTER(_Router), vp, i32, vp, vp, vp, vp, sz, vp]
         L.moin_route_static.argtypes = [ctypes.POINTER(_Router), vp, i32, vp, vp, vp, vp]
         L.moin_kmeans_update.argtypes = [ctypes.POINTER(_Plan), vp, vp, vp, vp, i32, vp]
+        L.moin_route_top2_workspace_bytes.restype = sz
+        L.moin_route_top2_workspace_bytes.argtypes = [i32, i32, i32]
+        L.moin_route_top2.argtypes = [ctypes.POINTER(_Router), vp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         L.moin_cache_create.argtypes = [i32, i32, ctypes.POINTER(_CacheProj), i32, vp, ctypes.POINTER(vp)]
         L.moin_cache_destroy.restype = None
         L.moin_cache_destroy.argtypes = [vp]
@@ -220,6 +223,21 @@ def route(router: Router, queries: torch.Tensor, out_expert: Optional[torch.Tens
     _check(lib().moin_route(ctypes.byref(router.c), _ptr(queries), Q, _ptr(out_expert), _ptr(out_centroid),
                             _ptr(out_best_sim), _ptr(ws), ws.numel(), _stream(stream)), "moin_route")
     return out_expert
+
+
+def route_top2(router: Router, queries: torch.Tensor, stream=None) -> dict:
+    """moin_route_top2: best centroid, runner-up and the margin between their cosines."""
+    assert queries.dtype == torch.bfloat16 and queries.dim() == 2 and queries.shape[1] == router.D
+    Q, dev = queries.shape[0], queries.device
+    out = {"expert": torch.empty(Q, dtype=torch.int32, device=dev), "centroid": torch.empty(Q, dtype=torch.int32, device=dev),
+           "second": torch.empty(Q, dtype=torch.int32, device=dev), "best": torch.empty(Q, dtype=torch.float32, device=dev),
+           "margin": torch.empty(Q, dtype=torch.float32, device=dev)}
+    n = lib().moin_route_top2_workspace_bytes(Q, router.K, router.D)
+    ws = torch.empty(max(n, 256), dtype=torch.uint8, device=dev)
+    _check(lib().moin_route_top2(ctypes.byref(router.c), _ptr(queries), Q, _ptr(out["expert"]), _ptr(out["centroid"]),
+                                 _ptr(out["second"]), _ptr(out["best"]), _ptr(out["margin"]), _ptr(ws), ws.numel(),
+                                 _stream(stream)), "moin_route_top2")
+    return out
 
 
 ROUTE_STATIC_MAX_Q = 65536

@@ -234,6 +234,55 @@ moin_status moin_route(const moin_router* router, const void* queries, int32_t Q
                                          out_centroid, out_best_sim, s));
 }
 
+size_t moin_route_top2_workspace_bytes(int32_t Q, int32_t K, int32_t D) {
+  (void)K; (void)D;
+  return 2 * align_up((size_t)(Q > 0 ? Q : 0) * sizeof(unsigned long long), 256) + 256;
+}
+
+moin_status moin_route_top2(const moin_router* router, const void* queries, int32_t Q, int32_t* out_expert,
+                            int32_t* out_centroid, int32_t* out_second, float* out_best_sim, float* out_margin,
+                            void* workspace, size_t workspace_bytes, moin_stream stream) {
+  if (!router || Q < 0) return MOIN_ERR_INVALID_ARG;
+  if (Q == 0) return MOIN_OK;
+  if (!queries || !router->centroids || !router->inv_norm || router->K < 1) return MOIN_ERR_INVALID_ARG;
+  const int K = router->K, D = router->D;
+  if (D < 8 || D > 8192 || (D % 8) != 0) return MOIN_ERR_BAD_SHAPE;
+  if (!aligned16(queries) || !aligned16(router->centroids)) return MOIN_ERR_MISALIGNED;
+  HostState* hs;
+  moin_status st = host_state(&hs);
+  if (st) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  const bool tc_ok = tc_router_supported(Q, K, D);
+  bool use_tc = tc_ok && (long long)Q * K >= (1ll << 16);
+  if (hs->gemm_impl == 1) use_tc = false;
+  if (hs->gemm_impl == 2) {
+    if (!tc_ok) return MOIN_ERR_BAD_SHAPE;
+    use_tc = true;
+  }
+  if (!use_tc) {
+    ProfScope prof(MOIN_K_ROUTE_SIMPLE, 1, s);
+    return record_cuda(launch_route_top2_simple((const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids,
+                                                router->inv_norm, router->centroid_to_expert, Q, K, D, out_expert,
+                                                out_centroid, out_second, out_best_sim, out_margin, s));
+  }
+  if (!workspace || workspace_bytes < moin_route_top2_workspace_bytes(Q, K, D) || !aligned16(workspace))
+    return MOIN_ERR_WORKSPACE;
+  const size_t half = align_up((size_t)Q * sizeof(unsigned long long), 256);
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(workspace);
+  unsigned long long* keys2 = reinterpret_cast<unsigned long long*>(reinterpret_cast<char*>(workspace) + half);
+  cudaError_t e = cudaMemsetAsync(workspace, 0, 2 * half, s);
+  if (e != cudaSuccess) return record_cuda(e);
+  {
+    ProfScope prof(MOIN_K_ROUTE_TC, 1, s);
+    st = launch_tc_router(hs, (const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids, router->inv_norm,
+                          Q, K, D, keys, s, keys2);
+  }
+  if (st) return st;
+  ProfScope prof(MOIN_K_ROUTE_FINISH, 1, s);
+  return record_cuda(launch_route_finish_top2(keys, keys2, (const __nv_bfloat16*)queries, router->centroid_to_expert, Q, D,
+                                              out_expert, out_centroid, out_second, out_best_sim, out_margin, s));
+}
+
 /* Scratch of moin_route_static: one 64-bit (similarity, index) key per query.  In host code the name
  * `g_route_static_keys` is only a handle for the runtime, not a device address; the address handed to
  * kernels comes from cudaGetSymbolAddress, looked up once per device. */

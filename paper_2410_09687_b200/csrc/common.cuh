@@ -135,6 +135,13 @@ cudaError_t launch_lora_expand_stream(const PlanView& pv, ExpandJobs jobs, float
                                       cudaStream_t stream);
 cudaError_t launch_gemm_warp(const __nv_bfloat16* x, const __nv_bfloat16* W, __nv_bfloat16* y, float* y0, int T,
                              int d_in, int d_out, cudaStream_t stream);
+cudaError_t launch_route_top2_simple(const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
+                                     const int* cmap, int Q, int K, int D, int* out_expert, int* out_centroid,
+                                     int* out_second, float* out_best, float* out_margin, cudaStream_t stream);
+cudaError_t launch_route_finish_top2(const unsigned long long* keys, const unsigned long long* keys2,
+                                     const __nv_bfloat16* q, const int* cmap, int Q, int D, int* out_expert,
+                                     int* out_centroid, int* out_second, float* out_best, float* out_margin,
+                                     cudaStream_t stream);
 cudaError_t launch_kmeans_mean(const PlanView& pv, const __nv_bfloat16* x, __nv_bfloat16* c_new, int D, int n_sms,
                                cudaStream_t stream);
 cudaError_t launch_inv_norm(const __nv_bfloat16* c, int K, int D, float* inv_norm, cudaStream_t stream);

@@ -408,6 +408,106 @@ cudaError_t launch_kmeans_mean(const PlanView& pv, const __nv_bfloat16* x, __nv_
   return cudaGetLastError();
 }
 
+// ----------------------------------------------------------------------------------------
+// Best and runner-up (top-2) router on the CUDA cores: one warp per query, lanes stride over the
+// embedding, centroids in increasing order (strict '>' keeps the lowest index among equals for both
+// places).  Small problems and odd shapes; the tensor-core path covers the rest.
+// ----------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+route_top2_simple_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ c,
+                         const float* __restrict__ inv_norm, const int* __restrict__ cmap, int Q, int K, int D,
+                         int* __restrict__ out_expert, int* __restrict__ out_centroid, int* __restrict__ out_second,
+                         float* __restrict__ out_best, float* __restrict__ out_margin) {
+  const int i = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (i >= Q) return;
+  const int nch = D / 8;
+  float best = -INFINITY, second = -INFINITY, qq = 0.f;
+  int best_k = 0, second_k = -1;
+  for (int k = 0; k < K; ++k) {
+    float acc = 0.f;
+    for (int ch = lane; ch < nch; ch += 32) {
+      const uint4 qv = ldg_cached(q + (size_t)i * D + ch * 8), cv = ldg_cached(c + (size_t)k * D + ch * 8);
+      const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w}, cw[4] = {cv.x, cv.y, cv.z, cv.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        acc = fmaf(bf16_lo(qw[e]), bf16_lo(cw[e]), acc);
+        acc = fmaf(bf16_hi(qw[e]), bf16_hi(cw[e]), acc);
+        if (k == 0) {
+          qq = fmaf(bf16_lo(qw[e]), bf16_lo(qw[e]), qq);
+          qq = fmaf(bf16_hi(qw[e]), bf16_hi(qw[e]), qq);
+        }
+      }
+    }
+    acc = warp_sum(acc);
+    const float inv = inv_norm[k];
+    const float sim = acc * inv;
+    if (inv > 0.f && sim > best) {
+      second = best; second_k = (best > -INFINITY) ? best_k : -1;
+      best = sim; best_k = k;
+    } else if (inv > 0.f && sim > second) {
+      second = sim; second_k = k;
+    }
+  }
+  qq = warp_sum(qq);
+  if (lane == 0) {
+    const float rq = rsqrtf(qq);
+    const int id = (best > -INFINITY) ? best_k : 0;
+    if (out_centroid) out_centroid[i] = id;
+    if (out_expert) out_expert[i] = cmap ? cmap[id] : id;
+    if (out_second) out_second[i] = (second > -INFINITY) ? second_k : -1;
+    if (out_best) out_best[i] = (best > -INFINITY) ? best * rq : -INFINITY;
+    if (out_margin) out_margin[i] = (second > -INFINITY) ? (best - second) * rq : INFINITY;
+  }
+}
+
+// Finishing pass of the tensor-core top-2 router: unpack both keys, divide by |q|.  One warp per query.
+__global__ void __launch_bounds__(256)
+route_finish_top2_kernel(const unsigned long long* __restrict__ keys, const unsigned long long* __restrict__ keys2,
+                         const __nv_bfloat16* __restrict__ q, const int* __restrict__ cmap, int Q, int D,
+                         int* __restrict__ out_expert, int* __restrict__ out_centroid, int* __restrict__ out_second,
+                         float* __restrict__ out_best, float* __restrict__ out_margin) {
+  const int i = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (i >= Q) return;
+  const unsigned long long k1 = keys[i], k2 = keys2[i];
+  float ss = 0.f;
+  for (int ch = lane; ch < D / 8; ch += 32) {
+    const uint4 v = ldg_cached(q + (size_t)i * D + ch * 8);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      ss = fmaf(bf16_lo(w[e]), bf16_lo(w[e]), ss);
+      ss = fmaf(bf16_hi(w[e]), bf16_hi(w[e]), ss);
+    }
+  }
+  ss = warp_sum(ss);
+  if (lane == 0) {
+    const float rq = rsqrtf(ss);
+    const int id = (k1 == 0ull) ? 0 : (int)(0xFFFFFFFFu - (uint32_t)(k1 & 0xFFFFFFFFull));
+    const float s1 = key_to_float((uint32_t)(k1 >> 32)), s2 = key_to_float((uint32_t)(k2 >> 32));
+    if (out_centroid) out_centroid[i] = id;
+    if (out_expert) out_expert[i] = cmap ? cmap[id] : id;
+    if (out_second) out_second[i] = (k2 == 0ull) ? -1 : (int)(0xFFFFFFFFu - (uint32_t)(k2 & 0xFFFFFFFFull));
+    if (out_best) out_best[i] = (k1 == 0ull) ? -INFINITY : s1 * rq;
+    if (out_margin) out_margin[i] = (k1 == 0ull || k2 == 0ull) ? INFINITY : (s1 - s2) * rq;
+  }
+}
+
+cudaError_t launch_route_top2_simple(const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
+                                     const int* cmap, int Q, int K, int D, int* out_expert, int* out_centroid,
+                                     int* out_second, float* out_best, float* out_margin, cudaStream_t stream) {
+  route_top2_simple_kernel<<<(Q + 7) / 8, 256, 0, stream>>>(q, c, inv_norm, cmap, Q, K, D, out_expert, out_centroid,
+                                                           out_second, out_best, out_margin);
+  return cudaGetLastError();
+}
+cudaError_t launch_route_finish_top2(const unsigned long long* keys, const unsigned long long* keys2,
+                                     const __nv_bfloat16* q, const int* cmap, int Q, int D, int* out_expert,
+                                     int* out_centroid, int* out_second, float* out_best, float* out_margin,
+                                     cudaStream_t stream) {
+  route_finish_top2_kernel<<<(Q + 7) / 8, 256, 0, stream>>>(keys, keys2, q, cmap, Q, D, out_expert, out_centroid, out_second,
+                                                           out_best, out_margin);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_inv_norm(const __nv_bfloat16* c, int K, int D, float* inv_norm, cudaStream_t stream) {
   centroid_inv_norm_kernel<<<(K + 7) / 8, 256, 0, stream>>>(c, K, D, inv_norm);
   return cudaGetLastError();

@@ -28,7 +28,7 @@ namespace moin {
 
 constexpr int kBM = 128, kBK = 64;
 constexpr int kTcThreads = 192;
-enum { EPI_STORE = 0, EPI_ROUTER = 1, EPI_SHRINK = 2 };
+enum { EPI_STORE = 0, EPI_ROUTER = 1, EPI_SHRINK = 2, EPI_ROUTER2 = 3 };   // ROUTER2: best and runner-up
 
 constexpr int kMaxShrinkJobs = 3;
 struct TcParams {
@@ -57,7 +57,8 @@ struct TcParams {
   __nv_bfloat16* ys[3];
   __nv_bfloat16* ys_lo[3];
   const float* inv_norm;       // EPI_ROUTER
-  unsigned long long* keys;    // EPI_ROUTER
+  unsigned long long* keys;    // EPI_ROUTER / EPI_ROUTER2: best (similarity, index) key per row
+  unsigned long long* keys2;   // EPI_ROUTER2: runner-up key per row
   DeviceStatus* status;
 };
 
@@ -242,6 +243,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const size_t grow = (size_t)(row0 + trow);
       float best = -INFINITY;
       int best_k = 0;
+      float second = -INFINITY;   // EPI_ROUTER2: runner-up of this tile's columns
+      int second_k = 0;
       const int ncols = (EPI == EPI_SHRINK) ? min(BN, (p.N + 31) / 32 * 32) : BN;
 #pragma unroll 1
       for (int c = 0; c < ncols; c += 32) {
@@ -249,7 +252,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint32_t v[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c, v);
         tmem_ld_wait();
-        if (EPI == EPI_ROUTER) {
+        if (EPI == EPI_ROUTER || EPI == EPI_ROUTER2) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             const int k = n0 + c + j;
@@ -257,8 +260,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               const float inv = __ldg(p.inv_norm + k);
               const float sim = __uint_as_float(v[j]) * inv;
               if (inv > 0.f && sim > best) {
+                if (EPI == EPI_ROUTER2) {
+                  second = best;
+                  second_k = best_k;
+                }
                 best = sim;
                 best_k = k;
+              } else if (EPI == EPI_ROUTER2 && inv > 0.f && sim > second) {
+                second = sim;
+                second_k = k;
               }
             }
           }
@@ -306,6 +316,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const unsigned long long key = ((unsigned long long)orderable(best) << 32) |
                                        (unsigned long long)(0xFFFFFFFFu - (uint32_t)best_k);
         atomicMax(p.keys + grow, key);
+      }
+      if (EPI == EPI_ROUTER2 && row_ok) {
+        // Two-slot merge: the max goes to keys; whatever loses a comparison there (the value it displaced, or
+        // the candidate itself) is offered to keys2.  Every candidate but the overall best is a loser exactly
+        // once, keys are distinct (they carry the index), and both slots are maxima: order independent.
+        const float cand[2] = {best, second};
+        const int cand_k[2] = {best_k, second_k};
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          if (cand[i] > -INFINITY) {
+            const unsigned long long key = ((unsigned long long)orderable(cand[i]) << 32) |
+                                           (unsigned long long)(0xFFFFFFFFu - (uint32_t)cand_k[i]);
+            const unsigned long long old = atomicMax(p.keys + grow, key);
+            const unsigned long long loser = old < key ? old : key;
+            if (loser != 0ull) atomicMax(p.keys2 + grow, loser);
+          }
+        }
       }
     }
   }
@@ -425,7 +452,8 @@ moin_status launch_tc_gemm(HostState* hs, const __nv_bfloat16* x, const __nv_bfl
 }
 
 moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
-                             int Q, int K, int D, unsigned long long* keys, cudaStream_t stream) {
+                             int Q, int K, int D, unsigned long long* keys, cudaStream_t stream,
+                             unsigned long long* keys2) {
   const long tiles_m = (Q + kBM - 1) / kBM;
   const int bn = pick_bn(tiles_m, K, hs->n_sms);
   CUtensorMap a, b;
@@ -433,8 +461,13 @@ moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_b
   if (!st) st = make_map(&b, c, K, D, bn);
   if (st) return st;
   TcParams p = {};
-  p.M = Q; p.N = K; p.K = D; p.inv_norm = inv_norm; p.keys = keys; p.status = hs->status;
+  p.M = Q; p.N = K; p.K = D; p.inv_norm = inv_norm; p.keys = keys; p.keys2 = keys2; p.status = hs->status;
   const long tiles = tiles_m * ((K + bn - 1) / bn);
+  if (keys2 != nullptr) {
+    if (bn == 256) return launch_cfg<256, EPI_ROUTER2>(hs, a, b, a, a, b, p, tiles, stream);
+    if (bn == 128) return launch_cfg<128, EPI_ROUTER2>(hs, a, b, a, a, b, p, tiles, stream);
+    return launch_cfg<64, EPI_ROUTER2>(hs, a, b, a, a, b, p, tiles, stream);
+  }
   if (bn == 256) return launch_cfg<256, EPI_ROUTER>(hs, a, b, a, a, b, p, tiles, stream);
   if (bn == 128) return launch_cfg<128, EPI_ROUTER>(hs, a, b, a, a, b, p, tiles, stream);
   return launch_cfg<64, EPI_ROUTER>(hs, a, b, a, a, b, p, tiles, stream);

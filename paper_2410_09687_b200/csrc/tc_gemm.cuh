@@ -20,7 +20,8 @@ moin_status launch_tc_gemm(HostState* hs, const __nv_bfloat16* x, const __nv_bfl
                            int T, int d_in, int d_out, cudaStream_t stream);
 // keys[i] = max over k of (orderable(<q_i,c_k> * inv_norm[k]) << 32 | (0xFFFFFFFF - k)), merged with atomicMax.
 moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
-                             int Q, int K, int D, unsigned long long* keys, cudaStream_t stream);
+                             int Q, int K, int D, unsigned long long* keys, cudaStream_t stream,
+                             unsigned long long* keys2 = nullptr);   // keys2 != nullptr: also the runner-up
 // Tile mode: hb = hi/lo bf16 parts of s * x A_e^T per row tile ([2][T][r]), then y = [x | hi | lo] [W ; B_e ; B_e]^T
 // in one GEMM.
 moin_status launch_tc_shrink_group(HostState* hs, const PlanView& pv, const moin_pool* const* pools,

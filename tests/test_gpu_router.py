@@ -116,3 +116,32 @@ def test_router_empty_batch():
     router = moin.Router(case.centroids.to(DEV))
     out = moin.route(router, torch.empty(0, 64, dtype=torch.bfloat16, device=DEV))
     assert out.numel() == 0
+
+
+@pytest.mark.parametrize("impl", [1, 2])   # 1: CUDA cores, 2: tcgen05 with the two-slot key merge
+@pytest.mark.parametrize("Q,K,D", [(300, 700, 768), (64, 1, 64), (1000, 5000, 128)])
+def test_router_runner_up_and_margin(impl, Q, K, D):
+    # best id as moin_route; the margin against the oracle's fp64 top-2 margin; the runner-up id is checked
+    # through its cosine (cos(second) = cos(best) - margin), since equal runners-up are all correct
+    case = mi.planted_router(K=K, Q=Q, D=D, seed=50 + K, unit_centroid_noise=True)
+    moin.set_option(moin.OPT_GEMM_IMPL, impl)
+    try:
+        router = moin.Router(case.centroids.to(DEV))
+        out = {k: v.cpu().numpy() for k, v in moin.route_top2(router, case.queries.to(DEV)).items()}
+    finally:
+        moin.set_option(moin.OPT_GEMM_IMPL, 0)
+    ref = _oracle(case)
+    assert_router_matches(out["centroid"], ref)
+    assert np.array_equal(out["expert"], out["centroid"])
+    np.testing.assert_allclose(out["best"], ref["best"], atol=2e-3)
+    if K == 1:
+        assert (out["second"] == -1).all() and np.isinf(out["margin"]).all()
+        return
+    tol = 2e-5 + 2e-3 * np.abs(ref["margin"])
+    assert (np.abs(out["margin"] - ref["margin"]) <= tol).all(), np.abs(out["margin"] - ref["margin"]).max()
+    c = mi.bf16_to_f64(case.centroids)
+    q = mi.bf16_to_f64(case.queries)
+    cos2 = (q * c[out["second"]]).sum(1) / (np.linalg.norm(q, axis=1) * np.linalg.norm(c[out["second"]], axis=1))
+    assert (np.abs(cos2 - (ref["best"] - ref["margin"])) <= tol).all()
+    assert (out["second"] != out["centroid"]).all()
+    assert moin.device_status()["timeout_flag"] == 0
