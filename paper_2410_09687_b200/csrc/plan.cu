@@ -97,24 +97,40 @@ __device__ __forceinline__ int block_incl_max(int v, int* smem) {
 }
 
 // Per expert id: exclusive prefix of its per-chunk counts over the chunks (in place) and the total.
-// One thread per expert id; counts are read in batches so the loads of a batch are in flight together.
-__global__ void __launch_bounds__(256) plan_prefix_kernel(PlanView v) {
-  const int k = blockIdx.x * 256 + threadIdx.x;
-  if (k > v.E) return;
+// A CTA covers 64 expert ids (threadIdx.x, so the loads of a chunk row are coalesced) and cuts the chunks into
+// kPrefixGroups consecutive ranges (threadIdx.y); a thread sums its range with its loads in flight in batches,
+// the ranges' totals meet in shared memory, and a second pass over the (now cached) counts writes the prefixes.
+constexpr int kPrefixIds = 64, kPrefixGroups = 4, kPrefixBatch = 16;
+__global__ void __launch_bounds__(kPrefixIds * kPrefixGroups) plan_prefix_kernel(PlanView v) {
+  __shared__ int s_sum[kPrefixGroups][kPrefixIds];
+  const int k = blockIdx.x * kPrefixIds + threadIdx.x, g = threadIdx.y;
+  const bool on = k <= v.E;
   const size_t pitch = (size_t)(v.E + 1);
+  const int per = (v.n_chunks + kPrefixGroups - 1) / kPrefixGroups;
+  const int c_lo = g * per, c_hi = min(v.n_chunks, c_lo + per);
+  int total = 0;
+  for (int c0 = c_lo; on && c0 < c_hi; c0 += kPrefixBatch) {
+    int n[kPrefixBatch];
+#pragma unroll
+    for (int j = 0; j < kPrefixBatch; ++j) n[j] = (c0 + j < c_hi) ? __ldcg(v.hist + (size_t)(c0 + j) * pitch + k) : 0;
+#pragma unroll
+    for (int j = 0; j < kPrefixBatch; ++j) total += n[j];
+  }
+  s_sum[g][threadIdx.x] = total;
+  __syncthreads();
   int run = 0;
-  constexpr int kBatch = 32;   // dependent round trips = chunks / kBatch
-  for (int c0 = 0; c0 < v.n_chunks; c0 += kBatch) {
-    int n[kBatch];
+  for (int gg = 0; gg < g; ++gg) run += s_sum[gg][threadIdx.x];
+  for (int c0 = c_lo; on && c0 < c_hi; c0 += kPrefixBatch) {
+    int n[kPrefixBatch];
 #pragma unroll
-    for (int j = 0; j < kBatch; ++j) n[j] = (c0 + j < v.n_chunks) ? __ldcg(v.hist + (size_t)(c0 + j) * pitch + k) : 0;
+    for (int j = 0; j < kPrefixBatch; ++j) n[j] = (c0 + j < c_hi) ? __ldcg(v.hist + (size_t)(c0 + j) * pitch + k) : 0;
 #pragma unroll
-    for (int j = 0; j < kBatch; ++j) {
-      if (c0 + j < v.n_chunks) v.hist[(size_t)(c0 + j) * pitch + k] = run;
+    for (int j = 0; j < kPrefixBatch; ++j) {
+      if (c0 + j < c_hi) v.hist[(size_t)(c0 + j) * pitch + k] = run;
       run += n[j];
     }
   }
-  v.keybase[k] = run;
+  if (on && g == kPrefixGroups - 1) v.keybase[k] = run;
 }
 
 // Row tiles: maximal runs of equal expert id in token order, cut every kTileRows rows.  One CTA of NT
@@ -313,7 +329,8 @@ cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, Device
   cudaError_t e = cudaMemsetAsync(v.hist, 0, sizeof(int) * (size_t)v.n_chunks * (size_t)(v.E + 1), stream);
   if (e != cudaSuccess) return e;
   plan_rank_kernel<<<v.n_chunks, kPlanChunk, 0, stream>>>(token_expert, v.T, v.E, v.key, v.rank, v.hist, status);
-  if (v.n_chunks > 1) plan_prefix_kernel<<<(v.E + 1 + 255) / 256, 256, 0, stream>>>(v);
+  if (v.n_chunks > 1)
+    plan_prefix_kernel<<<(v.E + 1 + kPrefixIds - 1) / kPrefixIds, dim3(kPrefixIds, kPrefixGroups), 0, stream>>>(v);
   plan_scan_kernel<<<1, 1024, 0, stream>>>(v, v.n_chunks > 1 ? 0 : 1, want_tiles);
   plan_scatter_kernel<<<v.n_chunks, kPlanChunk, 0, stream>>>(v);
   return cudaGetLastError();
