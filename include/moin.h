@@ -28,6 +28,10 @@
  *     hang: an out-of-range id means "no adapter" and is counted, a wait that runs out sets a
  *     flag, the kernel returns; both are read back with moin_device_status.
  *   - Results are deterministic: identical inputs give bit-identical outputs run to run.
+ *   - Devices and threads: the library keeps its host-side state (side streams, events, the address of the
+ *     status block, kernel attributes) per device ordinal and sets it up on the first call made with that
+ *     device current, so one process may drive several GPUs; calls that target the SAME device must come
+ *     from one host thread at a time (the per-device record and the side streams are not locked).
  *   - Arithmetic: bf16 operands, fp32 accumulation, one rounding to bf16 at the output.
  */
 #ifndef MOIN_H_
@@ -72,6 +76,16 @@ typedef struct {
 /* Copies the counters to *out (host).  SYNCHRONISES `stream`. */
 moin_status moin_device_status(moin_device_status_t* out, moin_stream stream);
 moin_status moin_device_status_reset(moin_stream stream);
+
+/* Self-test of the bounded wait (no counterpart in the paper).  Every device-side wait of the library gives up
+ * after a time limit instead of hanging; a healthy run never gets there.  This call launches one tiny kernel
+ * whose wait can never be satisfied (a barrier that nothing arms, no copy or MMA in flight) with a limit of
+ * limit_us microseconds (1..1 000 000), so that the expiry path runs: the wait returns, a second waiter leaves
+ * through the CTA's abort flag, the kernel ends normally, and moin_device_status afterwards shows timeout_flag
+ * != 0 with timeout_site = 99.  result (device, 3 x int32): [0] = 0 if the first wait gave up, [1] = 0 if the
+ * second waiter left through the abort flag, [2] = microseconds the kernel spent waiting.  Asynchronous on
+ * `stream`.  Call moin_device_status_reset afterwards. */
+moin_status moin_selftest_bounded_wait(int32_t limit_us, int32_t* result, moin_stream stream);
 
 /* Testing/tuning knobs (host-side path selection only; every path computes the same function).
  *   MOIN_OPT_GEMM_IMPL: 0 = automatic, 1 = force the warp-MMA kernels, 2 = force the tcgen05 kernels
@@ -147,13 +161,15 @@ moin_status moin_route_top2(const moin_router* router, const void* queries, int3
  * serving worker whose memory pool was sized and frozen at start-up, or a plug-in that runs inside
  * someone else's CUDA context and is forbidden to call cudaMalloc.)
  *
- * It computes exactly what moin_route computes, with the same arguments minus the workspace.  The
- * per-query scratch that the tensor-core router needs lives in a fixed array inside the library image
- * (MOIN_ROUTE_STATIC_MAX_Q * 8 bytes = 512 KiB, held by every GPU that loads the library until the
- * process exits).  The call performs no cudaMalloc/cudaFree and calls no allocating routine.
+ * It computes what moin_route computes - same arguments minus the workspace, same choice of kernel for the
+ * shape and the options in force, hence the same ids and the same cosines.  The per-query scratch that the
+ * tensor-core router needs lives in a fixed array inside the library image (MOIN_ROUTE_STATIC_MAX_Q * 8 bytes
+ * = 512 KiB, held by every GPU that loads the library until the process exits); shapes that moin_route serves
+ * without scratch do not touch it.  The call performs no cudaMalloc/cudaFree and calls no allocating routine.
  *   - Q > MOIN_ROUTE_STATIC_MAX_Q returns MOIN_ERR_WORKSPACE and launches nothing.
- *   - The first call on each device looks up the array's device address (with that device current);
- *     make that first call outside any stream capture.
+ *   - The first call on each device that needs the array looks up its device address (with that device
+ *     current); make that first call outside any stream capture, and from one host thread at a time (the
+ *     look-up is not guarded against two threads making their first call together).
  *   - All calls share the one array, which keeps the previous call's contents; the part a call uses is
  *     cleared on `stream` before use.  Two calls whose GPU work overlaps (different streams, no ordering
  *     between them) race on it: order them, or use moin_route with separate workspaces. */

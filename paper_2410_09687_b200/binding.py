@@ -24,6 +24,7 @@ EXPORTED_SYMBOLS = (
     "moin_decoder_workspace_bytes", "moin_decoder_forward", "moin_profile_enable", "moin_profile_read",
     "moin_kernel_name", "moin_route_static", "moin_lora_linear_group", "moin_lora_linear_group_workspace_bytes",
     "moin_kmeans_update", "moin_route_top2", "moin_route_top2_workspace_bytes", "moin_cache_create", "moin_cache_destroy", "moin_cache_admit", "moin_cache_slot_of",
+    "moin_selftest_bounded_wait",
 )
 
 
@@ -99,6 +100,7 @@ def lib() -> ctypes.CDLL:
         L.moin_device_status.argtypes = [ctypes.POINTER(_DevStatus), vp]
         L.moin_device_status_reset.argtypes = [vp]
         L.moin_set_option.argtypes = [i32, i32]
+        L.moin_selftest_bounded_wait.argtypes = [i32, vp, vp]
         L.moin_router_prepare.argtypes = [vp, i32, i32, vp, vp]
         L.moin_route_workspace_bytes.restype = sz
         L.moin_route_workspace_bytes.argtypes = [i32, i32, i32]
@@ -174,6 +176,15 @@ def device_status(stream=None) -> dict:
 
 def device_status_reset(stream=None) -> None:
     _check(lib().moin_device_status_reset(_stream(stream)), "moin_device_status_reset")
+
+
+def selftest_bounded_wait(limit_us: int, stream=None) -> dict:
+    """moin_selftest_bounded_wait: runs the expiry path of the library's bounded device-side wait once."""
+    res = torch.full((3,), -1, dtype=torch.int32, device="cuda")
+    _check(lib().moin_selftest_bounded_wait(int(limit_us), _ptr(res), _stream(stream)), "moin_selftest_bounded_wait")
+    torch.cuda.synchronize()
+    r = res.cpu().tolist()
+    return {"first_wait_returned_ok": r[0], "second_wait_returned_ok": r[1], "waited_us": r[2]}
 
 
 def profile_enable(capacity: int) -> None:

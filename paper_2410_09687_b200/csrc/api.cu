@@ -9,7 +9,8 @@ namespace moin {
 __device__ DeviceStatus g_device_status;
 
 static thread_local int t_last_cuda_error = 0;
-static HostState g_state;
+static HostState g_states[kMaxDevices];
+static int g_opt_gemm_impl = 0, g_opt_stream_impl = 0;   // moin_set_option: process-wide
 
 moin_status record_cuda(cudaError_t e) {
   if (e == cudaSuccess) return MOIN_OK;
@@ -21,6 +22,8 @@ moin_status host_state(HostState** out) {
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) { record_cuda(e); return MOIN_ERR_NO_DEVICE; }
+  if (dev < 0 || dev >= kMaxDevices) return MOIN_ERR_NO_DEVICE;
+  HostState& g_state = g_states[dev];
   if (g_state.device != dev) {
     cudaDeviceProp prop;
     e = cudaGetDeviceProperties(&prop, dev);
@@ -41,6 +44,8 @@ moin_status host_state(HostState** out) {
     g_state.n_sms = prop.multiProcessorCount;
     g_state.device = dev;
   }
+  g_state.gemm_impl = g_opt_gemm_impl;
+  g_state.stream_impl = g_opt_stream_impl;
   *out = &g_state;
   return MOIN_OK;
 }
@@ -95,11 +100,11 @@ int32_t moin_last_cuda_error(void) { return t_last_cuda_error; }
 
 moin_status moin_set_option(int32_t key, int32_t value) {
   if (key == MOIN_OPT_GEMM_IMPL && value >= 0 && value <= 2) {
-    g_state.gemm_impl = value;
+    g_opt_gemm_impl = value;
     return MOIN_OK;
   }
   if (key == MOIN_OPT_STREAM_IMPL && value >= 0 && value <= 2) {
-    g_state.stream_impl = value;
+    g_opt_stream_impl = value;
     return MOIN_OK;
   }
   return MOIN_ERR_INVALID_ARG;
@@ -186,19 +191,10 @@ size_t moin_route_workspace_bytes(int32_t Q, int32_t K, int32_t D) {
   return align_up((size_t)(Q > 0 ? Q : 0) * sizeof(unsigned long long), 256) + 256;
 }
 
-moin_status moin_route(const moin_router* router, const void* queries, int32_t Q, int32_t* out_expert,
-                       int32_t* out_centroid, float* out_best_sim, void* workspace, size_t workspace_bytes,
-                       moin_stream stream) {
-  if (!router || Q < 0) return MOIN_ERR_INVALID_ARG;
-  if (Q == 0) return MOIN_OK;
-  if (!queries || !out_expert || !router->centroids || !router->inv_norm || router->K < 1) return MOIN_ERR_INVALID_ARG;
-  const int K = router->K, D = router->D;
-  if (D < 8 || D > 8192 || (D % 8) != 0) return MOIN_ERR_BAD_SHAPE;
-  if (!aligned16(queries) || !aligned16(router->centroids)) return MOIN_ERR_MISALIGNED;
-  HostState* hs;
-  moin_status st = host_state(&hs);
-  if (st) return st;
-  cudaStream_t s = (cudaStream_t)stream;
+// Kernel choice shared by moin_route and moin_route_static, so that both compute the same values for the same
+// shapes and options: 0 = cluster kernel (decode-sized batch: one launch, no scratch), 1 = tensor-core GEMM with
+// one 64-bit key of scratch per query, 2 = CUDA-core kernel (no scratch).
+static moin_status route_choice(const HostState* hs, int Q, int K, int D, int* choice) {
   const bool tc_ok = tc_router_supported(Q, K, D);
   bool use_tc = tc_ok && (long long)Q * K >= (1ll << 16);
   if (hs->gemm_impl == 1) use_tc = false;
@@ -206,18 +202,26 @@ moin_status moin_route(const moin_router* router, const void* queries, int32_t Q
     if (!tc_ok) return MOIN_ERR_BAD_SHAPE;
     use_tc = true;
   }
-  if (hs->gemm_impl == 0 && route_cluster_supported(Q, K, D)) {   // decode-sized batch: one launch, no scratch
+  if (hs->gemm_impl == 0 && route_cluster_supported(Q, K, D)) *choice = 0;
+  else *choice = use_tc ? 1 : 2;
+  return MOIN_OK;
+}
+
+static moin_status route_launch(HostState* hs, int choice, const moin_router* router, const void* queries, int Q,
+                                int32_t* out_expert, int32_t* out_centroid, float* out_best_sim,
+                                unsigned long long* keys, cudaStream_t s) {
+  const int K = router->K, D = router->D;
+  if (choice == 0) {
     ProfScope prof(MOIN_K_ROUTE_CLUSTER, 1, s);
     return record_cuda(launch_route_cluster((const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids,
                                             router->inv_norm, router->centroid_to_expert, Q, K, D, out_expert,
                                             out_centroid, out_best_sim, s));
   }
-  if (use_tc) {
-    if (!workspace || workspace_bytes < moin_route_workspace_bytes(Q, K, D) || !aligned16(workspace))
-      return MOIN_ERR_WORKSPACE;
-    unsigned long long* keys = reinterpret_cast<unsigned long long*>(workspace);
+  if (choice == 1) {
+    // the merge across column tiles is a max, so the keys must start from zero
     cudaError_t e = cudaMemsetAsync(keys, 0, (size_t)Q * sizeof(unsigned long long), s);
     if (e != cudaSuccess) return record_cuda(e);
+    moin_status st;
     {
       ProfScope prof(MOIN_K_ROUTE_TC, 1, s);
       st = launch_tc_router(hs, (const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids,
@@ -232,6 +236,32 @@ moin_status moin_route(const moin_router* router, const void* queries, int32_t Q
   return record_cuda(launch_route_simple((const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids,
                                          router->inv_norm, router->centroid_to_expert, Q, K, D, out_expert,
                                          out_centroid, out_best_sim, s));
+}
+
+static moin_status route_check(const moin_router* router, const void* queries, int32_t Q, const int32_t* out_expert) {
+  if (!router || Q < 0) return MOIN_ERR_INVALID_ARG;
+  if (Q == 0) return MOIN_OK;
+  if (!queries || !out_expert || !router->centroids || !router->inv_norm || router->K < 1) return MOIN_ERR_INVALID_ARG;
+  const int D = router->D;
+  if (D < 8 || D > 8192 || (D % 8) != 0) return MOIN_ERR_BAD_SHAPE;
+  if (!aligned16(queries) || !aligned16(router->centroids)) return MOIN_ERR_MISALIGNED;
+  return MOIN_OK;
+}
+
+moin_status moin_route(const moin_router* router, const void* queries, int32_t Q, int32_t* out_expert,
+                       int32_t* out_centroid, float* out_best_sim, void* workspace, size_t workspace_bytes,
+                       moin_stream stream) {
+  moin_status st = route_check(router, queries, Q, out_expert);
+  if (st || Q == 0) return st;
+  HostState* hs;
+  if ((st = host_state(&hs))) return st;
+  int choice;
+  if ((st = route_choice(hs, Q, router->K, router->D, &choice))) return st;
+  if (choice == 1 && (!workspace || workspace_bytes < moin_route_workspace_bytes(Q, router->K, router->D) ||
+                      !aligned16(workspace)))
+    return MOIN_ERR_WORKSPACE;
+  return route_launch(hs, choice, router, queries, Q, out_expert, out_centroid, out_best_sim,
+                      reinterpret_cast<unsigned long long*>(workspace), (cudaStream_t)stream);
 }
 
 size_t moin_route_top2_workspace_bytes(int32_t Q, int32_t K, int32_t D) {
@@ -287,47 +317,29 @@ moin_status moin_route_top2(const moin_router* router, const void* queries, int3
  * `g_route_static_keys` is only a handle for the runtime, not a device address; the address handed to
  * kernels comes from cudaGetSymbolAddress, looked up once per device. */
 static __device__ __align__(256) unsigned long long g_route_static_keys[MOIN_ROUTE_STATIC_MAX_Q];
-static unsigned long long* g_route_static_ptr[64] = {nullptr};
+static unsigned long long* g_route_static_ptr[kMaxDevices] = {nullptr};
 
 moin_status moin_route_static(const moin_router* router, const void* queries, int32_t Q, int32_t* out_expert,
                               int32_t* out_centroid, float* out_best_sim, moin_stream stream) {
-  if (!router || Q < 0) return MOIN_ERR_INVALID_ARG;
-  if (Q == 0) return MOIN_OK;
+  moin_status st = route_check(router, queries, Q, out_expert);
+  if (st || Q == 0) return st;
   if (Q > MOIN_ROUTE_STATIC_MAX_Q) return MOIN_ERR_WORKSPACE;   // beyond the built-in scratch
-  if (!queries || !out_expert || !router->centroids || !router->inv_norm || router->K < 1) return MOIN_ERR_INVALID_ARG;
-  const int K = router->K, D = router->D;
-  if (D < 8 || D > 8192 || (D % 8) != 0) return MOIN_ERR_BAD_SHAPE;
-  if (!aligned16(queries) || !aligned16(router->centroids)) return MOIN_ERR_MISALIGNED;
   HostState* hs;
-  moin_status st = host_state(&hs);
-  if (st) return st;
-  cudaStream_t s = (cudaStream_t)stream;
-  if (!tc_router_supported(Q, K, D)) {   // tiny embedding dimension: the CUDA-core kernel needs no scratch
-    ProfScope prof(MOIN_K_ROUTE_SIMPLE, 1, s);
-    return record_cuda(launch_route_simple((const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids,
-                                           router->inv_norm, router->centroid_to_expert, Q, K, D, out_expert,
-                                           out_centroid, out_best_sim, s));
+  if ((st = host_state(&hs))) return st;
+  int choice;
+  if ((st = route_choice(hs, Q, router->K, router->D, &choice))) return st;
+  unsigned long long* keys = nullptr;
+  if (choice == 1) {   // only the tensor-core kernel needs scratch
+    if (g_route_static_ptr[hs->device] == nullptr) {   // set-up: once per device, that device is current here
+      void* p = nullptr;
+      cudaError_t e = cudaGetSymbolAddress(&p, g_route_static_keys);
+      if (e != cudaSuccess) return record_cuda(e);
+      g_route_static_ptr[hs->device] = reinterpret_cast<unsigned long long*>(p);
+    }
+    keys = g_route_static_ptr[hs->device];   // still holds the previous call's keys: route_launch clears Q of them
   }
-  if (hs->device < 0 || hs->device >= 64) return MOIN_ERR_NO_DEVICE;
-  if (g_route_static_ptr[hs->device] == nullptr) {   // set-up: once per device, that device is current here
-    void* p = nullptr;
-    cudaError_t e = cudaGetSymbolAddress(&p, g_route_static_keys);
-    if (e != cudaSuccess) return record_cuda(e);
-    g_route_static_ptr[hs->device] = reinterpret_cast<unsigned long long*>(p);
-  }
-  unsigned long long* keys = g_route_static_ptr[hs->device];
-  // the array still holds the previous call's keys: the merge is a max, so it must start from zero
-  cudaError_t e = cudaMemsetAsync(keys, 0, (size_t)Q * sizeof(unsigned long long), s);
-  if (e != cudaSuccess) return record_cuda(e);
-  {
-    ProfScope prof(MOIN_K_ROUTE_TC, 1, s);
-    st = launch_tc_router(hs, (const __nv_bfloat16*)queries, (const __nv_bfloat16*)router->centroids,
-                          router->inv_norm, Q, K, D, keys, s);
-  }
-  if (st) return st;
-  ProfScope prof(MOIN_K_ROUTE_FINISH, 1, s);
-  return record_cuda(launch_route_finish(keys, (const __nv_bfloat16*)queries, router->centroid_to_expert, Q, D,
-                                         out_expert, out_centroid, out_best_sim, s));
+  return route_launch(hs, choice, router, queries, Q, out_expert, out_centroid, out_best_sim, keys,
+                      (cudaStream_t)stream);
 }
 
 /* ------------------------------------------------------------------ K-means update */

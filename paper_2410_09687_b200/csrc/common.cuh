@@ -155,19 +155,41 @@ cudaError_t launch_route_cluster(const __nv_bfloat16* q, const __nv_bfloat16* c,
 cudaError_t launch_route_finish(const unsigned long long* keys, const __nv_bfloat16* q, const int* cmap, int Q, int D,
                                 int* out_expert, int* out_centroid, float* out_best, cudaStream_t stream);
 
-// Process-wide host state shared by the entry points (api.cu).
+// Host state of the entry points (api.cu): one record per device ordinal, filled on the first call made with
+// that device current.  Streams, events, the status block's address and the kernels' shared-memory opt-ins all
+// belong to one device, so nothing here is shared between devices.
+constexpr int kMaxDevices = 64;
+constexpr int kOptinSlots = 48;
 struct HostState {
   DeviceStatus* status = nullptr;  // device address of the status block
   int device = -1;
   int n_sms = 0;
-  int gemm_impl = 0;               // MOIN_OPT_GEMM_IMPL
+  int gemm_impl = 0;               // MOIN_OPT_GEMM_IMPL (process-wide option, copied in on every call)
   int stream_impl = 0;             // MOIN_OPT_STREAM_IMPL
   // fork/join inside one call: independent kernels of a call run on `side` between two events
   cudaStream_t side[kMaxStreamJobs] = {nullptr, nullptr, nullptr, nullptr};
   cudaEvent_t ev_fork = nullptr, ev_join[kMaxStreamJobs] = {nullptr, nullptr, nullptr, nullptr};
+  size_t smem_optin[kOptinSlots] = {};   // dynamic shared memory already opted in, per kernel (see ensure_smem_optin)
 };
 moin_status host_state(HostState** out);      // lazily initialised for the current device
 moin_status record_cuda(cudaError_t e);       // MOIN_OK or MOIN_ERR_CUDA (remembers e)
+
+// Kernels that need more than 48 KB of dynamic shared memory opt in with cudaFuncSetAttribute; the driver keeps
+// that attribute per device, so the "already done" note is kept per device too (slot = one id per kernel).
+enum {
+  OPTIN_TC_GEMM = 0,        // + 4 * (BN index) + EPI, 12 entries; + 12 for the short-ring instantiations
+  OPTIN_ROUTE_CLUSTER = 24, OPTIN_ROUTE_SIMPLE = 25, OPTIN_SHRINK_TMA = 26, OPTIN_EXPAND_TMA = 27,
+  OPTIN_LORA_FUSED = 28, OPTIN_ATTENTION = 29, OPTIN_ROUTE_PLAN = 30
+};
+template <class Fn>
+inline cudaError_t ensure_smem_optin(int slot, Fn* fn, size_t bytes) {
+  HostState* hs = nullptr;
+  if (host_state(&hs) != MOIN_OK) return cudaErrorInvalidDevice;
+  if (hs->smem_optin[slot] >= bytes) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) hs->smem_optin[slot] = bytes;
+  return e;
+}
 
 // Brackets the launches issued during its lifetime with two CUDA events when profiling is enabled.
 struct ProfScope {

@@ -449,13 +449,9 @@ moin_status launch_lora_shrink_tma(HostState* hs, const PlanView& pv, const moin
   // stage layout: 4 box slots of 64 rows (8 KB each) + 8 token rows, the same for every projection of the launch
   const int stage_bytes = (int)align_up((size_t)4 * 64 * 128 + 8 * kSXPitch, 1024);
   const int stages = pick_stages(ring_bytes, stage_bytes);
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(lora_shrink_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-    if (e != cudaSuccess) return record_cuda(e);
-    configured = true;
-  }
-  cudaError_t e = cudaMemsetAsync(queue, 0, sizeof(int), stream);
+  cudaError_t e = ensure_smem_optin(OPTIN_SHRINK_TMA, lora_shrink_tma_kernel, 220 * 1024);
+  if (e != cudaSuccess) return record_cuda(e);
+  e = cudaMemsetAsync(queue, 0, sizeof(int), stream);
   if (e != cudaSuccess) return record_cuda(e);
   const int grid = (int)(items < hs->n_sms ? (items < 1 ? 1 : items) : hs->n_sms);
   lora_shrink_tma_kernel<<<grid, kShrinkThreads, ring_smem(stages, stage_bytes), stream>>>(
@@ -485,13 +481,9 @@ moin_status launch_lora_expand_tma(HostState* hs, const PlanView& pv, const moin
     }
   }
   const int stages = pick_stages(ring_bytes, kEStageBytes);
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(lora_expand_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-    if (e != cudaSuccess) return record_cuda(e);
-    configured = true;
-  }
-  cudaError_t e = cudaMemsetAsync(queue, 0, sizeof(int), stream);
+  cudaError_t e = ensure_smem_optin(OPTIN_EXPAND_TMA, lora_expand_tma_kernel, 220 * 1024);
+  if (e != cudaSuccess) return record_cuda(e);
+  e = cudaMemsetAsync(queue, 0, sizeof(int), stream);
   if (e != cudaSuccess) return record_cuda(e);
   const int grid = (int)(items < hs->n_sms ? (items < 1 ? 1 : items) : hs->n_sms);
   lora_expand_tma_kernel<<<grid, kExpandThreads, ring_smem(stages, kEStageBytes), stream>>>(

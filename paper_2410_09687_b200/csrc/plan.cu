@@ -238,7 +238,7 @@ template <int NT>   // threads = sort width: the power of two at or above T, at 
 __global__ void __launch_bounds__(NT) plan_small_kernel(const int* __restrict__ token_expert, PlanView v,
                                                         DeviceStatus* status, int want_tiles) {
   __shared__ int s_key[NT];        // sanitised id by token
-  __shared__ int s_sort[NT];       // sort keys, then the segment starts
+  __shared__ int s_sort[NT + 1];   // sort keys, then the segment starts plus one end marker (NT segments at most)
   __shared__ int s_row0[NT + 1];   // tile starts
   __shared__ int smem[33];
   __shared__ int s_carry[2];

@@ -35,7 +35,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceStatus* st,
-                                          int site) {
+                                          int site, unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   unsigned long long t0 = 0;
   uint32_t spins = 0;
@@ -44,7 +44,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const unsigned long long now = global_ns();
       if (t0 == 0) t0 = now;
-      if (now - t0 > kWaitLimitNs) {
+      if (now - t0 > limit_ns) {
         *abort_flag = 1;
         atomicExch(&st->timeout_flag, 1);
         atomicExch(&st->timeout_site, site);

@@ -332,12 +332,8 @@ cudaError_t launch_route_cluster(const __nv_bfloat16* q, const __nv_bfloat16* c,
                                  const int* cmap, int Q, int K, int D, int* out_expert, int* out_centroid,
                                  float* out_best, cudaStream_t stream) {
   const size_t smem = (size_t)kRcQ * (D * 2 + 16);
-  static size_t configured = 0;
-  if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(route_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
+  cudaError_t ce = ensure_smem_optin(OPTIN_ROUTE_CLUSTER, route_cluster_kernel, smem);
+  if (ce != cudaSuccess) return ce;
   const int groups = (Q + kRcQ - 1) / kRcQ;
   route_cluster_kernel<<<groups * kRcCluster, kRcWarps * 32, smem, stream>>>(q, c, inv_norm, cmap, Q, K, D, out_expert,
                                                                             out_centroid, out_best);
@@ -517,12 +513,8 @@ cudaError_t launch_route_simple(const __nv_bfloat16* q, const __nv_bfloat16* c, 
                                 const int* cmap, int Q, int K, int D, int* out_expert, int* out_centroid,
                                 float* out_best, cudaStream_t stream) {
   const size_t smem = (size_t)kRouteQB * D * 2;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(route_simple_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 8192 * 2);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  cudaError_t ce = ensure_smem_optin(OPTIN_ROUTE_SIMPLE, route_simple_kernel, 8 * 8192 * 2);
+  if (ce != cudaSuccess) return ce;
   route_simple_kernel<<<(Q + kRouteQB - 1) / kRouteQB, 128, smem, stream>>>(q, c, inv_norm, cmap, Q, K, D, out_expert,
                                                                             out_centroid, out_best);
   return cudaGetLastError();

@@ -390,13 +390,9 @@ static moin_status launch_cfg(HostState* hs, const CUtensorMap& a, const CUtenso
                               const CUtensorMap& a3, const CUtensorMap& b2, const TcParams& p, long max_tiles,
                               cudaStream_t stream, const CUtensorMap* b3 = nullptr) {
   using Cfg = TcCfg<BN>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)Cfg::kSmemBytes);
-    if (e != cudaSuccess) return record_cuda(e);
-    configured = true;
-  }
+  constexpr int slot = OPTIN_TC_GEMM + 4 * (BN == 256 ? 2 : BN == 128 ? 1 : 0) + EPI;
+  cudaError_t e = ensure_smem_optin(slot, tc_gemm_kernel<BN, EPI>, Cfg::kSmemBytes);
+  if (e != cudaSuccess) return record_cuda(e);
   long grid = max_tiles < hs->n_sms ? max_tiles : hs->n_sms;
   if (grid < 1) grid = 1;
   tc_gemm_kernel<BN, EPI><<<(int)grid, kTcThreads, Cfg::kSmemBytes, stream>>>(a, b, a2, a3, b2, b3 ? *b3 : b2, p);

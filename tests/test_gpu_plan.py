@@ -79,6 +79,22 @@ def test_plan_single_launch_and_chunked_paths_at_the_switch():
     _check(np.repeat(rng.integers(0, 3, size=4), 256).astype(np.int32), 3)   # runs longer than one tile
 
 
+def test_plan_all_distinct_at_every_sort_width():
+    # T equal to the single-launch sort width with every token on its own expert: as many segments as the
+    # sort has slots, so the end marker of the segment list sits one past the last sort slot
+    for T in (128, 256, 512, 1024):
+        for mode in (moin.PLAN_SEGMENTS, moin.PLAN_TILES):
+            te = np.arange(T, dtype=np.int32)
+            plan = moin.plan_build(torch.from_numpy(te).to(DEV), T, mode)
+            got = plan.read()
+            assert got["S"] == T
+            assert np.array_equal(got["perm"], te) and np.array_equal(got["seg_expert"], te)
+            assert np.array_equal(got["seg_start"], np.arange(T + 1))
+            if mode == moin.PLAN_TILES:
+                assert got["n_tiles"] == T and np.array_equal(got["tile_expert"], te)
+        _check(np.arange(T, dtype=np.int32)[::-1].copy(), T)
+
+
 def test_plan_is_deterministic():
     rng = np.random.default_rng(4)
     te = torch.from_numpy(rng.integers(0, 100, size=5000).astype(np.int32)).to(DEV)
