@@ -90,7 +90,8 @@ moin_status moin_selftest_bounded_wait(int32_t limit_us, int32_t* result, moin_s
 /* Testing/tuning knobs (host-side path selection only; every path computes the same function).
  *   MOIN_OPT_GEMM_IMPL: 0 = automatic, 1 = force the warp-MMA kernels, 2 = force the tcgen05 kernels
  *                       (calls whose shapes the forced kernel cannot take fail with MOIN_ERR_BAD_SHAPE). */
-/*   MOIN_OPT_STREAM_IMPL: short-segment LoRA kernels: 0 = automatic, 1 = register-fed kernels, 2 = TMA-staged kernels. */
+/*   MOIN_OPT_STREAM_IMPL: short-segment LoRA kernels: 0 = automatic (the fused launch), 1 = separate shrink and
+ *   expand launches beside base GEMMs on side streams, 2 = TMA-staged kernels, 3 = fused shrink + expand launch. */
 enum { MOIN_OPT_GEMM_IMPL = 1, MOIN_OPT_STREAM_IMPL = 2 };
 moin_status moin_set_option(int32_t key, int32_t value);
 
@@ -107,7 +108,8 @@ typedef struct {
 enum {
   MOIN_K_ROUTE_SIMPLE = 0, MOIN_K_ROUTE_TC = 1, MOIN_K_ROUTE_FINISH = 2, MOIN_K_PLAN = 3, MOIN_K_GEMM_WARP = 4,
   MOIN_K_GEMM_TC = 5, MOIN_K_SHRINK_STREAM = 6, MOIN_K_EXPAND_STREAM = 7, MOIN_K_SHRINK_TC = 8,
-  MOIN_K_FUSED_TC = 9, MOIN_K_GLUE = 10, MOIN_K_ATTENTION = 11, MOIN_K_ROUTE_CLUSTER = 12, MOIN_K_KMEANS_UPDATE = 13, MOIN_K_COUNT = 14
+  MOIN_K_FUSED_TC = 9, MOIN_K_GLUE = 10, MOIN_K_ATTENTION = 11, MOIN_K_ROUTE_CLUSTER = 12, MOIN_K_KMEANS_UPDATE = 13,
+  MOIN_K_FUSED_STREAM = 14, MOIN_K_COUNT = 15
 };
 moin_status moin_profile_enable(int32_t capacity);
 moin_status moin_profile_read(moin_profile_record* out, int32_t capacity, int32_t* n);

@@ -21,8 +21,10 @@
  * benchmark's CPU-baseline leg use it.
  *
  * Pins (tests that tie this file to something other than itself) are in
- * tests/test_oracle_*.py; the decoder's absolute logits have no external pin
- * ("parity unpinned" beyond the structural pins listed there).
+ * tests/test_oracle_*.py.  Every function has one: the decoder's exact variant is held
+ * against the `transformers` Llama implementation in float64 (base model, and each routed
+ * request with its adapter merged into the weights), and its storage-rounded variant against
+ * a numpy restatement of one block that rounds at exactly the listed points.
  */
 #include <math.h>
 #include <stdint.h>

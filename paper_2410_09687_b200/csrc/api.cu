@@ -103,7 +103,7 @@ moin_status moin_set_option(int32_t key, int32_t value) {
     g_opt_gemm_impl = value;
     return MOIN_OK;
   }
-  if (key == MOIN_OPT_STREAM_IMPL && value >= 0 && value <= 2) {
+  if (key == MOIN_OPT_STREAM_IMPL && value >= 0 && value <= 3) {
     g_opt_stream_impl = value;
     return MOIN_OK;
   }
@@ -169,7 +169,8 @@ moin_status moin_profile_read(moin_profile_record* out, int32_t capacity, int32_
 const char* moin_kernel_name(int32_t k) {
   static const char* names[MOIN_K_COUNT] = {"route_simple", "route_tc", "route_finish", "plan", "gemm_warp", "gemm_tc",
                                             "lora_shrink_stream", "lora_expand_stream", "lora_shrink_tc",
-                                            "lora_fused_tc", "decoder_glue", "attention", "route_cluster", "kmeans_update"};
+                                            "lora_fused_tc", "decoder_glue", "attention", "route_cluster", "kmeans_update",
+                                            "lora_fused_stream"};
   return (k >= 0 && k < MOIN_K_COUNT) ? names[k] : "unknown";
 }
 
@@ -571,6 +572,52 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
     parts[j] = tma_stream ? lora_stream_parts(d_in[j]) : 1;
     h[j] = reinterpret_cast<float*>(ws_job[j]);   // [parts][T][r] (partial) shrink results
     y0[j] = reinterpret_cast<float*>(ws_job[j] + align_up((size_t)lora_stream_parts(d_in[j]) * (size_t)T * (size_t)r[j] * sizeof(float), 256));
+  }
+  if (!tma_stream && hs->stream_impl != 1) {
+    // One stream, programmatic dependent launches: the base GEMMs first (projections with the same d_in share a
+    // launch), then ONE launch that holds the shrink items and the expand CTAs of the whole group.  The fused
+    // launch starts beside the GEMMs (its shrink items do not depend on them); its expand CTAs wait for them.
+    {
+      ProfScope prof(MOIN_K_GEMM_TC, 1, s);
+      for (int j0 = 0; j0 < n_jobs;) {
+        if (!use_tc[j0]) {
+          if ((st = record_cuda(launch_gemm_warp(xs[j0], (const __nv_bfloat16*)jobs[j0].W, ys[j0], y0[j0], T, d_in[j0],
+                                                 d_out[j0], s))))
+            return st;
+          ++j0;
+          continue;
+        }
+        const __nv_bfloat16* gw[kTcMaxStoreJobs];
+        int gd[kTcMaxStoreJobs], n = 0;
+        while (j0 + n < n_jobs && n < kTcMaxStoreJobs && use_tc[j0 + n] && d_in[j0 + n] == d_in[j0]) {
+          gw[n] = (const __nv_bfloat16*)jobs[j0 + n].W;
+          gd[n] = d_out[j0 + n];
+          ++n;
+        }
+        if ((st = launch_tc_gemm_group(hs, xs + j0, gw, ys + j0, y0 + j0, gd, n, T, d_in[j0], s))) return st;
+        j0 += n;
+      }
+    }
+    ShrinkJobs sj = {};
+    ExpandJobs ej = {};
+    sj.n = ej.n = n_jobs;
+    for (int j = 0; j < n_jobs; ++j) {
+      sj.x[j] = xs[j];
+      sj.A[j] = (const __nv_bfloat16*)jobs[j].pool->A;
+      sj.h[j] = h[j];
+      sj.slot_of_expert[j] = jobs[j].pool->slot_of_expert;
+      sj.r[j] = r[j];
+      sj.d_in[j] = d_in[j];
+      ej.h[j] = h[j];
+      ej.B[j] = (const __nv_bfloat16*)jobs[j].pool->B;
+      ej.y0[j] = y0[j];
+      ej.y[j] = ys[j];
+      ej.slot_of_expert[j] = jobs[j].pool->slot_of_expert;
+      ej.r[j] = r[j];
+      ej.d_out[j] = d_out[j];
+    }
+    ProfScope prof(MOIN_K_FUSED_STREAM, 1, s);
+    return record_cuda(launch_lora_fused_stream(pv, sj, ej, scale, hs->n_sms, hs->status, s));
   }
   cudaError_t ce = cudaEventRecord(hs->ev_fork, s);
   if (ce != cudaSuccess) return record_cuda(ce);

@@ -18,6 +18,12 @@ bool tc_fused_supported(int r);
 // y = x W^T (bf16) and optionally y0 = x W^T (fp32).
 moin_status launch_tc_gemm(HostState* hs, const __nv_bfloat16* x, const __nv_bfloat16* W, __nv_bfloat16* y, float* y0,
                            int T, int d_in, int d_out, cudaStream_t stream);
+// The same for up to kTcMaxStoreJobs projections that share T and d_in, in one launch that takes part in
+// programmatic dependent launch (waits for the kernel before it, lets the kernel after it start beside it).
+constexpr int kTcMaxStoreJobs = 3;
+moin_status launch_tc_gemm_group(HostState* hs, const __nv_bfloat16* const* xs, const __nv_bfloat16* const* Ws,
+                                 __nv_bfloat16* const* ys, float* const* y0s, const int* d_outs, int n_jobs, int T,
+                                 int d_in, cudaStream_t stream);
 // keys[i] = max over k of (orderable(<q_i,c_k> * inv_norm[k]) << 32 | (0xFFFFFFFF - k)), merged with atomicMax.
 moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
                              int Q, int K, int D, unsigned long long* keys, cudaStream_t stream,

@@ -37,9 +37,9 @@ def test_tiny_config_routed_by_the_router():
     assert_layer_close(y, oracle_layer(case), "tiny routed")
 
 
-@pytest.fixture(params=[1, 2], ids=["regfed", "tma"])
+@pytest.fixture(params=[1, 2, 3], ids=["two-launch", "tma", "fused"])
 def stream_impl(request):
-    """Both implementations of the short-segment kernels (register-fed and TMA-staged)."""
+    """Every implementation of the short-segment kernels (separate shrink / expand launches, TMA-staged, fused launch)."""
     moin.set_option(moin.OPT_STREAM_IMPL, request.param)
     yield request.param
     moin.set_option(moin.OPT_STREAM_IMPL, 0)
