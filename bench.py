@@ -279,7 +279,12 @@ class LayerWorkload:
             flops += 2.0 * T * d_in * d_out + 2.0 * T * r * (d_in + d_out)
         step_bytes = sum((d_out * d_in + T * d_in + T * d_out + n_distinct * r * (d_in + d_out)) * 2
                          for _, d_in, d_out in self.projs) + self.R * self.D * 2 + self.K * self.D * 2
-        return {"per_kernel_bytes": per, "step_bytes": step_bytes, "step_flops": flops}
+        # long-run mode: the fused GEMM's own work is the base product plus hi and lo K blocks of the rank
+        rb = (r + 63) // 64 * 64
+        fused = sum(2.0 * T * d_out * (d_in + 2 * rb) for _, d_in, d_out in self.projs)
+        shrink_tc = sum(2.0 * T * r * d_in for _, d_in, d_out in self.projs)
+        return {"per_kernel_bytes": per, "step_bytes": step_bytes, "step_flops": flops,
+                "per_kernel_flops": {"lora_fused_tc": fused, "lora_shrink_tc": shrink_tc}}
 
     def config(self) -> dict:
         name = (f"decode: 7 TinyLlama projections, 500 experts rank {self.r}, 256 single tokens, router 256x500x768"
@@ -550,6 +555,10 @@ def timed_loop(world, fn, steps: int, warmup: int, use_graph: bool) -> float:
     return e0.elapsed_time(e1) / steps, graphs is not None
 
 
+def wl_cache_free(wl) -> bool:
+    return getattr(wl, "cache", None) is None
+
+
 def profile_pass(moin, fn, steps: int):
     """Per-kernel device time (CUDA events inside the library, on the launching stream)."""
     moin.profile_enable(65536)
@@ -571,6 +580,146 @@ def profile_pass(moin, fn, steps: int):
         a["launches"] += r["launches"]; a["brackets"] += 1; a["ms"] += r["ms"]
     launches_per_step = sum(a["launches"] for a in agg.values()) / steps
     return agg, launches_per_step
+
+
+def kernel_timeline(fn, use_graph: bool, steps: int = 6):
+    """Start / end of every kernel of one step, from the profiler's activity records of `steps` replays (the
+    kernels keep running concurrently while they are recorded).  Returns (rows, span_us) for the median-length
+    step: rows = [(name, start_us, end_us)] relative to the step's first kernel.  None if no records come back."""
+    try:
+        from torch.profiler import ProfilerActivity, profile
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            graphs = []
+            for i in range(ROTATE):
+                fn(i)
+            stream.synchronize()
+            if use_graph:
+                for i in range(ROTATE):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=stream):
+                        fn(i)
+                    graphs.append(g)
+            run = (lambda i: graphs[i % ROTATE].replay()) if use_graph else fn
+            for i in range(ROTATE):
+                run(i)
+            stream.synchronize()
+            with profile(activities=[ProfilerActivity.CUDA]) as prof:
+                for i in range(steps + 1):
+                    run(i)
+                stream.synchronize()
+        evs = sorted((e for e in prof.events() if e.device_type == torch.autograd.DeviceType.CUDA and "moin::" in e.name),
+                     key=lambda e: e.time_range.start)
+        if not evs:
+            return None
+        first = evs[0].name
+        cuts = [i for i, e in enumerate(evs) if e.name == first]
+        if len(cuts) < 3:
+            return None
+        spans = [(evs[cuts[k + 1]].time_range.start - evs[cuts[k]].time_range.start, k) for k in range(len(cuts) - 1)]
+        span, k = sorted(spans)[len(spans) // 2]
+        t0 = evs[cuts[k]].time_range.start
+        rows = [(e.name, e.time_range.start - t0, e.time_range.end - t0) for e in evs[cuts[k]:cuts[k + 1]]]
+        return rows, span
+    except Exception as e:  # pragma: no cover
+        sys.stderr.write(f"[bench] no kernel timeline ({e})\n")
+        return None
+
+
+def critical_path(rows, span_us: float) -> dict:
+    """Where a step's time goes, from its kernel timeline.  Kernels on the call's own stream follow one another, so
+    their durations add up; the base GEMMs of the short-segment path run on side streams beside the shrink, and
+    only the part of a GEMM that outlasts the shrink it runs beside delays the expand ("gemm_exposed").  The
+    remainder of the step is launch gaps.  No entry can exceed the step."""
+    def short(n):
+        n = n.split("moin::")[1].split("(")[0].split("<")[0]
+        return n.replace("_kernel", "")
+    main, side = {}, []
+    ordered = sorted(rows, key=lambda r: r[1])
+    for name, a, b in ordered:
+        k = short(name)
+        if k.startswith("tc_gemm") or k.startswith("gemm_warp"):
+            side.append((a, b))
+        else:
+            main[k] = main.get(k, 0.0) + (b - a)
+    exposed = 0.0
+    if side and any(k.startswith("lora_expand") for k in main):
+        # per expand launch: how long after the end of the shrink before it did the last GEMM before it end?
+        exp = [(a, b) for n, a, b in ordered if "lora_expand" in n]
+        shr = [(a, b) for n, a, b in ordered if "lora_shrink" in n]
+        for (ea, _), (_, sb) in zip(exp, shr):
+            g_end = max([b for a, b in side if a < ea] or [0.0])
+            exposed += max(0.0, min(g_end, ea) - sb)
+        out = dict(main)
+        out["gemm_exposed"] = exposed
+    else:   # everything on one stream
+        out = dict(main)
+        for a, b in side:
+            out["tc_gemm"] = out.get("tc_gemm", 0.0) + (b - a)
+    out = {k: round(v, 2) for k, v in out.items()}
+    out["gaps"] = round(max(0.0, span_us - sum(out.values())), 2)
+    out["step_us"] = round(span_us, 2)
+    return out
+
+
+def tensor_roofline(top: str, a: dict, alg: dict, prof_steps: int, peaks: dict, kind: str) -> dict:
+    """Roofline object of a long-run tensor-core kernel: ITS OWN flops per launch over its own launch time
+    (CUDA-event brackets, the kernel alone between them), against the burst peak a kernel timed in isolation sees."""
+    fl = alg["per_kernel_flops"][top] * prof_steps / a["launches"]
+    sec = a["ms"] * 1e-3 / a["launches"]
+    ach = fl / sec / 1e12
+    return {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+            "frac": ach / peaks["bf16_tflops"], "frac_sustained": ach / peaks["bf16_tflops_sustained"],
+            "frac_nominal": ach / NOMINAL_BF16_TFLOPS, "peak_source": peaks["source"] + " (burst)",
+            "algorithmic_flops_per_launch": fl, "avg_launch_ms": sec * 1e3, "traffic": traffic_for(top, kind)}
+
+
+def side_prefill(moin, dev: str, peaks: dict, local: int) -> dict:
+    """Prefill workload (32 x 512 tokens, 5000 rank-16 experts) as an extra key of the default line."""
+    wl = LayerWorkload("prefill", dev)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, graphed = timed_loop(1, wl.step, 400, 5, True)     # >= 0.5 s of timed work
+    clocks = sampler.stop()
+    agg, _ = profile_pass(moin, wl.step, 10)
+    nd = wl.distinct()
+    alg = wl.algorithmic(nd)
+    t_tc = alg["step_flops"] / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = alg["step_bytes"] / (peaks["hbm_gbs"] * 1e9)
+    out = {"workload": wl.config()["workload"], "ms_per_step": ms, "tokens_per_s": wl.T / (ms * 1e-3),
+           "launch": "cuda_graph replay" if graphed else "plain launches", "clocks": clocks,
+           "step_roofline": {"bound": "tensor" if t_tc >= t_hbm else "hbm", "roofline_ms": max(t_tc, t_hbm) * 1e3,
+                             "frac": max(t_tc, t_hbm) * 1e3 / ms,
+                             "frac_nominal": max(alg["step_flops"] / (NOMINAL_BF16_TFLOPS * 1e12),
+                                                 alg["step_bytes"] / (NOMINAL_HBM_GBS * 1e9)) * 1e3 / ms,
+                             "peak": "burst"},
+           "distinct_experts": nd}
+    if "lora_fused_tc" in agg:
+        out["roofline"] = tensor_roofline("lora_fused_tc", agg["lora_fused_tc"], alg, 10, peaks, "prefill")
+    out["kernels"] = {k: {"launches": a["launches"], "ms_per_launch": a["ms"] / max(a["launches"], 1)} for k, a in agg.items()}
+    del wl
+    torch.cuda.empty_cache()
+    return out
+
+
+def side_forward(moin, dev: str, peaks: dict, local: int) -> dict:
+    """Full decoder forward (22 blocks, 64 x 256 tokens, 500 rank-64 experts) as an extra key of the default line."""
+    wl = ForwardWorkload(dev)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, _ = timed_loop(1, wl.step, 14, 3, False)           # >= 0.5 s of timed work
+    clocks = sampler.stop()
+    alg = wl.algorithmic()
+    ach = alg["flops"] / (ms * 1e-3) / 1e12
+    out = {"workload": wl.config()["workload"], "ms_per_step": ms, "tokens_per_s": wl.T / (ms * 1e-3), "clocks": clocks,
+           "achieved_tflops": ach, "frac": ach / peaks["bf16_tflops_sustained"], "peak": "sustained",
+           "frac_burst": ach / peaks["bf16_tflops"], "frac_nominal": ach / NOMINAL_BF16_TFLOPS,
+           "algorithmic_flops": alg["flops"]}
+    del wl
+    torch.cuda.empty_cache()
+    return out
 
 
 def traffic_for(kernel: str, workload: str):
@@ -674,13 +823,13 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-router-extra", action="store_true")
+    ap.add_argument("--no-side-workloads", action="store_true", help="decode line without the prefill / forward keys")
     ap.add_argument("--forward-layers", type=int, default=22)
     ap.add_argument("--no-group", action="store_true", help="one moin_lora_linear call per projection")
     ap.add_argument("--cache-slots", type=int, default=None,
                     help="decode / prefill through the two-tier adapter store with this many device slots (side "
                          "measurement: the step then contains a host round trip and the copies of the missing adapters)")
     ap.add_argument("--rank", type=int, default=None, help="decode / prefill at another LoRA rank than the config's (side measurement)")
-    ap.add_argument("--stream-impl", type=int, default=0, help="short-segment LoRA kernels: 0 auto, 1 register-fed, 2 TMA-staged")
     args = ap.parse_args()
     defaults = {"decode": (3000, 20), "prefill": (100, 5), "router": (50, 5), "forward": (5, 3), "kmeans": (50, 5)}
     if args.impl == "reference":
@@ -697,7 +846,6 @@ def main():
         from paper_2410_09687_b200 import build
         build.build()
     moin.lib()
-    moin.set_option(moin.OPT_STREAM_IMPL, args.stream_impl)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
     world, rank, local = dist_setup(args.gpus)
@@ -740,9 +888,9 @@ def main():
     # (decode) path the base GEMMs run on side streams beside the shrink, so their brackets overlap it
     on_path = {k: v for k, v in agg.items() if not (kind == "decode" and k in ("gemm_tc", "gemm_warp"))}
     top = max(on_path.items(), key=lambda kv: kv[1]["ms"])[0]
-    total_ms = sum(a["ms"] for a in agg.values())
-    kernels = {k: {"launches": a["launches"], "ms_per_launch": a["ms"] / max(a["launches"], 1),
-                   "share": a["ms"] / total_ms} for k, a in agg.items()}
+    kernels = {k: {"launches": a["launches"], "ms_per_launch": a["ms"] / max(a["launches"], 1)} for k, a in agg.items()}
+    tl = kernel_timeline(wl.step, use_graph) if (rank == 0 and kind != "forward" and wl_cache_free(wl)) else None
+    path = critical_path(*tl) if tl else None
     prof_steps = min(args.steps, 20)
     roof = None
     extra = {}
@@ -773,14 +921,7 @@ def main():
                     "algorithmic_bytes_per_launch": bytes_per_launch, "avg_launch_ms": sec * 1e3,
                     "traffic": traffic_for(top, kind)}
         elif top in ("lora_fused_tc", "lora_shrink_tc"):
-            a = agg[top]
-            fl = alg["step_flops"] * prof_steps / a["launches"]
-            sec = a["ms"] * 1e-3 / a["launches"]
-            ach = fl / sec / 1e12
-            roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
-                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "frac_burst": ach / peaks["bf16_tflops"],
-                    "frac_nominal": ach / NOMINAL_BF16_TFLOPS, "peak_source": peaks["source"] + " (sustained)",
-                    "algorithmic_flops_per_launch": fl, "avg_launch_ms": sec * 1e3, "traffic": traffic_for(top, kind)}
+            roof = tensor_roofline(top, agg[top], alg, prof_steps, peaks, kind)
     elif kind in ("router", "kmeans"):
         alg = wl.algorithmic()
         a = agg[top]
@@ -847,6 +988,10 @@ def main():
         m = moin.route_top2(wl.router, rq)["margin"]
         extra["near_ties"] = {"margin_below": 1e-4, "count": int((m < 1e-4).sum().item()), "of": int(rq.shape[0]),
                               "min_margin": float(m.min().item())}
+    if kind == "decode" and rank == 0 and world == 1 and not args.no_side_workloads and wl.cache is None and not args.rank:
+        # the other headline workloads, so that one line carries all of them (their own runs: --workload ...)
+        extra["prefill"] = side_prefill(moin, dev, peaks, local)
+        extra["forward"] = side_forward(moin, dev, peaks, local)
     if rank == 0:
         metric = {"router": "router_queries_per_s", "kmeans": "kmeans_points_per_s"}.get(kind, "routed_lora_tokens_per_s")
         cfg = wl.config()
@@ -859,7 +1004,7 @@ def main():
                         "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h, "ms_per_step": ms_e2e,
                         "pipelining": e2e_mode},
                 "gpu_launches": int(round(launches_per_step * args.steps)), "roofline": roof, "kernels": kernels,
-                "cpu_baseline": cpu}
+                "critical_path_us": path, "cpu_baseline": cpu}
         line.update(extra)
         print(json.dumps(line), flush=True)
     if world > 1:

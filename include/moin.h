@@ -90,9 +90,7 @@ moin_status moin_selftest_bounded_wait(int32_t limit_us, int32_t* result, moin_s
 /* Testing/tuning knobs (host-side path selection only; every path computes the same function).
  *   MOIN_OPT_GEMM_IMPL: 0 = automatic, 1 = force the warp-MMA kernels, 2 = force the tcgen05 kernels
  *                       (calls whose shapes the forced kernel cannot take fail with MOIN_ERR_BAD_SHAPE). */
-/*   MOIN_OPT_STREAM_IMPL: short-segment LoRA kernels: 0 = automatic (the fused launch), 1 = separate shrink and
- *   expand launches beside base GEMMs on side streams, 2 = TMA-staged kernels, 3 = fused shrink + expand launch. */
-enum { MOIN_OPT_GEMM_IMPL = 1, MOIN_OPT_STREAM_IMPL = 2 };
+enum { MOIN_OPT_GEMM_IMPL = 1 };
 moin_status moin_set_option(int32_t key, int32_t value);
 
 /* Per-kernel timing for benchmarks (no counterpart in the paper).  While enabled, every kernel group the
@@ -108,8 +106,7 @@ typedef struct {
 enum {
   MOIN_K_ROUTE_SIMPLE = 0, MOIN_K_ROUTE_TC = 1, MOIN_K_ROUTE_FINISH = 2, MOIN_K_PLAN = 3, MOIN_K_GEMM_WARP = 4,
   MOIN_K_GEMM_TC = 5, MOIN_K_SHRINK_STREAM = 6, MOIN_K_EXPAND_STREAM = 7, MOIN_K_SHRINK_TC = 8,
-  MOIN_K_FUSED_TC = 9, MOIN_K_GLUE = 10, MOIN_K_ATTENTION = 11, MOIN_K_ROUTE_CLUSTER = 12, MOIN_K_KMEANS_UPDATE = 13,
-  MOIN_K_FUSED_STREAM = 14, MOIN_K_COUNT = 15
+  MOIN_K_FUSED_TC = 9, MOIN_K_GLUE = 10, MOIN_K_ATTENTION = 11, MOIN_K_ROUTE_CLUSTER = 12, MOIN_K_KMEANS_UPDATE = 13, MOIN_K_COUNT = 14
 };
 moin_status moin_profile_enable(int32_t capacity);
 moin_status moin_profile_read(moin_profile_record* out, int32_t capacity, int32_t* n);
@@ -376,6 +373,18 @@ moin_status moin_decoder_forward(const moin_model* model, const int32_t* tokens,
                                  const int32_t* req_expert, int32_t R, int32_t T, int32_t max_seqlen,
                                  void* logits, int32_t logits_mode, const moin_decoder_taps* taps,
                                  void* workspace, size_t workspace_bytes, moin_stream stream);
+
+/* The same forward with one expert id per TOKEN: token_expert [T] int32, device, -1 = base only for that token.
+ * Paper Sec. 5 (future work: "per-token adapters"); Sec. 3.3 itself uses one expert per request, which is the case
+ * token_expert[t] = req_expert[request of t] and gives bit-identical results to moin_decoder_forward.  Every
+ * projection of every block applies, row by row, the adapter of that row's token; attention, norms and the MLP
+ * are unchanged.  The run structure of the ids is not known to the host, so the call reads the batch plan's
+ * header back once (it synchronises `stream` once, before the first block).  All other arguments, layouts and
+ * errors as for moin_decoder_forward; token_expert == NULL is MOIN_ERR_INVALID_ARG. */
+moin_status moin_decoder_forward_per_token(const moin_model* model, const int32_t* tokens, const int32_t* cu_seqlens,
+                                           const int32_t* token_expert, int32_t R, int32_t T, int32_t max_seqlen,
+                                           void* logits, int32_t logits_mode, const moin_decoder_taps* taps,
+                                           void* workspace, size_t workspace_bytes, moin_stream stream);
 
 #ifdef __cplusplus
 }

@@ -62,9 +62,14 @@ def lib() -> ctypes.CDLL:
                                                                      ctypes.c_int64, ctypes.c_int,
                                                                      ctypes.c_int64, ctypes.c_int64,
                                                                      ctypes.c_double, ctypes.c_void_p]
+        L.moin_oracle_lora_linear_ex.restype = ctypes.c_int
+        L.moin_oracle_lora_linear_ex.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                                                        ctypes.c_void_p, ctypes.c_int, ctypes.c_int64,
+                                                                        ctypes.c_int64, ctypes.c_int, ctypes.c_int64,
+                                                                        ctypes.c_int64, ctypes.c_double, ctypes.c_void_p]
         L.moin_oracle_decoder_forward.restype = ctypes.c_int
         L.moin_oracle_decoder_forward.argtypes = [ctypes.POINTER(_Model), ctypes.c_void_p, ctypes.c_void_p,
-                                                  ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64,
+                                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64,
                                                   ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.moin_oracle_bucket.restype = ctypes.c_int64
@@ -134,9 +139,15 @@ def route(q: np.ndarray, c: np.ndarray, centroid_to_expert: Optional[np.ndarray]
     return {"centroid": cid, "expert": eid, "best": best, "margin": margin}
 
 
+ACT_NONE, ACT_RELU, ACT_SILU, ACT_GELU = 0, 1, 2, 3
+
+
 def lora_linear(x: np.ndarray, W: np.ndarray, A: Optional[np.ndarray], B: Optional[np.ndarray],
-                token_expert: Optional[np.ndarray], slot_of_expert: Optional[np.ndarray], scale: float) -> np.ndarray:
-    """y[T, d_out] (float64) of the routed LoRA layer; A [n_slots, r, d_in], B [n_slots, d_out, r]."""
+                token_expert: Optional[np.ndarray], slot_of_expert: Optional[np.ndarray], scale: float,
+                slot_rank: Optional[np.ndarray] = None, act: int = ACT_NONE) -> np.ndarray:
+    """y[T, d_out] (float64) of the routed LoRA layer; A [n_slots, r, d_in], B [n_slots, d_out, r].
+    ``slot_rank`` ([n_slots] int32): rank of each slot's adapter (<= r; rows of A / columns of B beyond it are
+    not read); ``act``: function applied between the two low-rank matrices."""
     (x, W, A, B), kind = _same_kind(x, W, A, B)
     T, d_in = x.shape
     d_out = W.shape[0]
@@ -150,8 +161,15 @@ def lora_linear(x: np.ndarray, W: np.ndarray, A: Optional[np.ndarray], B: Option
         assert int(so.max()) < A.shape[0]
     E = 0 if so is None else so.shape[0]
     y = np.zeros((T, d_out), np.float64)
-    rc = lib().moin_oracle_lora_linear(_ptr(x), _ptr(W), _ptr(A), _ptr(B), kind, _ptr(te), _ptr(so), T, E, r,
-                                       d_in, d_out, float(scale), _ptr(y))
+    if slot_rank is None and act == ACT_NONE:
+        rc = lib().moin_oracle_lora_linear(_ptr(x), _ptr(W), _ptr(A), _ptr(B), kind, _ptr(te), _ptr(so), T, E, r,
+                                           d_in, d_out, float(scale), _ptr(y))
+    else:
+        sr = None if slot_rank is None else np.ascontiguousarray(slot_rank, dtype=np.int32)
+        if sr is not None and A is not None:
+            assert sr.shape[0] == A.shape[0]
+        rc = lib().moin_oracle_lora_linear_ex(_ptr(x), _ptr(W), _ptr(A), _ptr(B), kind, _ptr(te), _ptr(so), _ptr(sr),
+                                              int(act), T, E, r, d_in, d_out, float(scale), _ptr(y))
     if rc:
         raise RuntimeError(f"moin_oracle_lora_linear failed: {rc}")
     return y
@@ -242,7 +260,9 @@ class DecoderOracle:
 
     def forward(self, tokens, cu_seqlens, req_expert, layer_begin: int = 0, layer_end: Optional[int] = None,
                 round_storage: bool = False, hidden_in: Optional[np.ndarray] = None,
-                want_hidden: bool = False, want_logits: bool = True):
+                want_hidden: bool = False, want_logits: bool = True, token_expert=None):
+        """``token_expert`` ([T] int32): one expert per token instead of one per request (the paper's
+        future-work variant, Sec. 5); ``req_expert`` is then ignored."""
         cfg = self.cfg
         layer_end = cfg.n_layers if layer_end is None else layer_end
         tokens = np.ascontiguousarray(tokens, dtype=np.int32)
@@ -252,7 +272,8 @@ class DecoderOracle:
         hin = None if hidden_in is None else np.ascontiguousarray(hidden_in, dtype=np.float64)
         hout = np.zeros((T, cfg.hidden), np.float64) if want_hidden else None
         logits = np.zeros((T, cfg.vocab), np.float64) if want_logits else None
-        rc = lib().moin_oracle_decoder_forward(ctypes.byref(self._m), _ptr(tokens), _ptr(cu), _ptr(re_), R, T,
+        te_ = None if token_expert is None else np.ascontiguousarray(token_expert, dtype=np.int32)
+        rc = lib().moin_oracle_decoder_forward(ctypes.byref(self._m), _ptr(tokens), _ptr(cu), _ptr(re_), _ptr(te_), R, T,
                                                layer_begin, layer_end, int(round_storage), _ptr(hin),
                                                _ptr(hout), _ptr(logits))
         if rc:

@@ -148,9 +148,37 @@ int moin_oracle_route(const void* q, const void* c, int dtype, int64_t Q, int64_
  *                                      if slot >= 0)
  * y is left in double.  One token per loop iteration; tokens are independent.
  * ------------------------------------------------------------------------------------ */
+/* Optional function between the two low-rank matrices (the paper's formula has none; Sec. 5 lists "an
+ * activation between the two LoRA matrices" as a variant): y = W x + s W_b act(W_a x). */
+#define ORACLE_ACT_NONE 0
+#define ORACLE_ACT_RELU 1
+#define ORACLE_ACT_SILU 2
+#define ORACLE_ACT_GELU 3
+static double activate(double v, int act) {
+  switch (act) {
+    case ORACLE_ACT_RELU: return v > 0.0 ? v : 0.0;
+    case ORACLE_ACT_SILU: return v / (1.0 + exp(-v));
+    case ORACLE_ACT_GELU: return 0.5 * v * (1.0 + erf(v / sqrt(2.0)));
+    default: return v;
+  }
+}
+
+/* r = rows of A / columns of B STORED per slot; r_use <= r = how many of them this slot's adapter has (the
+ * paper's future-work "adaptive rank", Sec. 5: a rank per topic; Sec. 4 trains all at one rank, r_use = r).
+ * Entries beyond r_use are never read. */
+static void lora_token_ex(const void* x, size_t xoff, int xdtype, const void* W, const void* A,
+                          const void* B, int wdtype, int64_t slot, int r, int r_use, int act, int64_t d_in,
+                          int64_t d_out, double s, double* y /* [d_out] */, double* h /* [r] */);
+
 static void lora_token(const void* x, size_t xoff, int xdtype, const void* W, const void* A,
                        const void* B, int wdtype, int64_t slot, int r, int64_t d_in,
                        int64_t d_out, double s, double* y /* [d_out] */, double* h /* [r] */) {
+  lora_token_ex(x, xoff, xdtype, W, A, B, wdtype, slot, r, r, ORACLE_ACT_NONE, d_in, d_out, s, y, h);
+}
+
+static void lora_token_ex(const void* x, size_t xoff, int xdtype, const void* W, const void* A,
+                          const void* B, int wdtype, int64_t slot, int r, int r_use, int act, int64_t d_in,
+                          int64_t d_out, double s, double* y /* [d_out] */, double* h /* [r] */) {
   for (int64_t j = 0; j < d_out; ++j) {
     double acc = 0.0;
     for (int64_t i = 0; i < d_in; ++i)
@@ -158,17 +186,17 @@ static void lora_token(const void* x, size_t xoff, int xdtype, const void* W, co
     y[j] = acc;
   }
   if (slot < 0 || A == NULL || B == NULL) return;
-  for (int p = 0; p < r; ++p) {
+  for (int p = 0; p < r_use; ++p) {
     double acc = 0.0;
     size_t base = ((size_t)slot * (size_t)r + (size_t)p) * (size_t)d_in;
     for (int64_t i = 0; i < d_in; ++i)
       acc += ld(A, wdtype, base + (size_t)i) * ld(x, xdtype, xoff + (size_t)i);
-    h[p] = acc;
+    h[p] = activate(acc, act);
   }
   for (int64_t j = 0; j < d_out; ++j) {
     double acc = 0.0;
     size_t base = ((size_t)slot * (size_t)d_out + (size_t)j) * (size_t)r;
-    for (int p = 0; p < r; ++p) acc += ld(B, wdtype, base + (size_t)p) * h[p];
+    for (int p = 0; p < r_use; ++p) acc += ld(B, wdtype, base + (size_t)p) * h[p];
     y[j] += s * acc;
   }
 }
@@ -176,6 +204,31 @@ static void lora_token(const void* x, size_t xoff, int xdtype, const void* W, co
 static int64_t slot_for(const int32_t* slot_of_expert, int64_t E, int32_t e) {
   if (e < 0 || e >= E || slot_of_expert == NULL) return -1;
   return slot_of_expert[e];
+}
+
+/* slot_rank (nullable, [n_slots]): rank of each slot's adapter, at most r; NULL = every slot has rank r.
+ * act: ORACLE_ACT_*. */
+int moin_oracle_lora_linear_ex(const void* x, const void* W, const void* A, const void* B, int dtype,
+                               const int32_t* token_expert, const int32_t* slot_of_expert,
+                               const int32_t* slot_rank, int act,
+                               int64_t T, int64_t E, int r, int64_t d_in, int64_t d_out, double s,
+                               double* y /* [T][d_out] */) {
+  if (T < 0 || d_in <= 0 || d_out <= 0 || r < 0 || act < 0 || act > ORACLE_ACT_GELU) return -1;
+#pragma omp parallel
+  {
+    double* h = (double*)malloc(sizeof(double) * (size_t)(r > 0 ? r : 1));
+#pragma omp for schedule(dynamic, 1)
+    for (int64_t t = 0; t < T; ++t) {
+      int64_t slot = token_expert ? slot_for(slot_of_expert, E, token_expert[t]) : -1;
+      int r_use = (slot >= 0 && slot_rank) ? slot_rank[slot] : r;
+      if (r_use > r) r_use = r;
+      if (r_use < 0) r_use = 0;
+      lora_token_ex(x, (size_t)t * (size_t)d_in, dtype, W, A, B, dtype, slot, r, r_use, act, d_in, d_out, s,
+                    y + (size_t)t * (size_t)d_out, h);
+    }
+    free(h);
+  }
+  return 0;
 }
 
 int moin_oracle_lora_linear(const void* x, const void* W, const void* A, const void* B, int dtype,
@@ -240,16 +293,18 @@ static void rmsnorm(const double* v, const uint16_t* gain, int n, double eps, in
   for (int i = 0; i < n; ++i) out[i] = maybe_round(v[i] * inv * ld(gain, ORACLE_BF16, (size_t)i), rnd);
 }
 
-/* One projection of one request: rows [0, L) of in[L][d_in] -> out[L][d_out]. */
+/* One projection of one request: rows [0, L) of in[L][d_in] -> out[L][d_out]; slots[t] = adapter slot of
+ * token t (-1: base only).  The paper uses one expert per request (Sec. 3.3: slots all equal); an expert per
+ * token is its future-work variant (Sec. 5) and needs nothing but a slot per row. */
 static void project(const moin_oracle_model* m, int layer, int proj, const double* in, int64_t L,
-                    int64_t d_in, int64_t d_out, int64_t slot, int rnd, double* out, double* h) {
+                    int64_t d_in, int64_t d_out, const int64_t* slots, int rnd, double* out, double* h) {
   const void* W = m->W[layer * 7 + proj];
   const void* A = m->A ? m->A[layer * 7 + proj] : NULL;
   const void* B = m->B ? m->B[layer * 7 + proj] : NULL;
   for (int64_t t = 0; t < L; ++t) {
     /* activations are doubles here; weights are bf16 */
     double* y = out + (size_t)t * (size_t)d_out;
-    lora_token(in, (size_t)t * (size_t)d_in, ORACLE_F64, W, A, B, ORACLE_BF16, slot, m->r, d_in,
+    lora_token(in, (size_t)t * (size_t)d_in, ORACLE_F64, W, A, B, ORACLE_BF16, slots[t], m->r, d_in,
                d_out, m->scale, y, h);
     if (rnd)
       for (int64_t j = 0; j < d_out; ++j) y[j] = round_bf16(y[j]);
@@ -273,7 +328,7 @@ static void rope_inplace(double* v /* [L][n_h*hd] */, int64_t L, int n_h, int hd
 
 /* Blocks [layer_begin, layer_end) applied to one request's residual stream xr[L][hidden]. */
 static int run_blocks(const moin_oracle_model* m, int layer_begin, int layer_end, double* xr,
-                      int64_t L, int64_t slot, int rnd) {
+                      int64_t L, const int64_t* slot, int rnd) {
   const int H = m->hidden, nh = m->n_heads, nkv = m->n_kv_heads, hd = m->head_dim, F = m->ffn;
   const int qd = nh * hd, kvd = nkv * hd, group = nh / nkv;
   size_t LL = (size_t)L;
@@ -349,7 +404,8 @@ static int run_blocks(const moin_oracle_model* m, int layer_begin, int layer_end
  *   logits     (nullable) [T][vocab] double: final norm + lm_head (only meaningful when
  *              layer_end == n_layers). */
 int moin_oracle_decoder_forward(const moin_oracle_model* m, const int32_t* tokens,
-                                const int32_t* cu_seqlens, const int32_t* req_expert, int32_t R,
+                                const int32_t* cu_seqlens, const int32_t* req_expert,
+                                const int32_t* token_expert, int32_t R,
                                 int64_t T, int layer_begin, int layer_end, int round_storage,
                                 const double* hidden_in, double* hidden_out, double* logits) {
   if (!m || R < 0 || T < 0 || layer_begin < 0 || layer_end > m->n_layers || layer_begin > layer_end)
@@ -360,9 +416,14 @@ int moin_oracle_decoder_forward(const moin_oracle_model* m, const int32_t* token
   for (int32_t rq = 0; rq < R; ++rq) {
     int64_t t0 = cu_seqlens[rq], L = cu_seqlens[rq + 1] - cu_seqlens[rq];
     if (L <= 0) continue;
-    int64_t slot = req_expert ? slot_for(m->slot_of_expert, m->E, req_expert[rq]) : -1;
+    /* adapter slot of every token: the request's expert (Sec. 3.3), or the token's own if token_expert is given */
+    int64_t* slot = (int64_t*)malloc(sizeof(int64_t) * (size_t)L);
     double* xr = (double*)malloc(sizeof(double) * (size_t)L * (size_t)H);
-    if (!xr) { rc = -2; continue; }
+    if (!xr || !slot) { rc = -2; free(xr); free(slot); continue; }
+    for (int64_t t = 0; t < L; ++t) {
+      if (token_expert) slot[t] = slot_for(m->slot_of_expert, m->E, token_expert[t0 + t]);
+      else slot[t] = req_expert ? slot_for(m->slot_of_expert, m->E, req_expert[rq]) : -1;
+    }
     for (int64_t t = 0; t < L; ++t)
       for (int i = 0; i < H; ++i)
         xr[(size_t)t * H + i] = hidden_in ? hidden_in[(size_t)(t0 + t) * H + i]
@@ -384,6 +445,7 @@ int moin_oracle_decoder_forward(const moin_oracle_model* m, const int32_t* token
       free(xn);
     }
     free(xr);
+    free(slot);
   }
   return rc;
 }

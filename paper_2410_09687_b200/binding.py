@@ -15,7 +15,6 @@ _lib: Optional[ctypes.CDLL] = None
 PLAN_AUTO, PLAN_SEGMENTS, PLAN_TILES = 0, 1, 2
 LOGITS_ALL, LOGITS_LAST, LOGITS_NONE = 0, 1, 2
 OPT_GEMM_IMPL = 1
-OPT_STREAM_IMPL = 2
 
 EXPORTED_SYMBOLS = (
     "moin_status_string", "moin_version", "moin_last_cuda_error", "moin_device_status", "moin_device_status_reset",
@@ -24,7 +23,7 @@ EXPORTED_SYMBOLS = (
     "moin_decoder_workspace_bytes", "moin_decoder_forward", "moin_profile_enable", "moin_profile_read",
     "moin_kernel_name", "moin_route_static", "moin_lora_linear_group", "moin_lora_linear_group_workspace_bytes",
     "moin_kmeans_update", "moin_route_top2", "moin_route_top2_workspace_bytes", "moin_cache_create", "moin_cache_destroy", "moin_cache_admit", "moin_cache_slot_of",
-    "moin_selftest_bounded_wait",
+    "moin_selftest_bounded_wait", "moin_decoder_forward_per_token",
 )
 
 
@@ -130,6 +129,7 @@ def lib() -> ctypes.CDLL:
         L.moin_decoder_workspace_bytes.argtypes = [ctypes.POINTER(_Model), i32, i32]
         L.moin_decoder_forward.argtypes = [ctypes.POINTER(_Model), vp, vp, vp, i32, i32, i32, vp, i32,
                                            ctypes.POINTER(_Taps), vp, sz, vp]
+        L.moin_decoder_forward_per_token.argtypes = L.moin_decoder_forward.argtypes
         L.moin_profile_enable.argtypes = [i32]
         L.moin_profile_read.argtypes = [ctypes.POINTER(_ProfRec), i32, ctypes.POINTER(i32)]
         L.moin_kernel_name.restype = ctypes.c_char_p
@@ -494,8 +494,9 @@ def decoder_forward(model: DecoderModel, tokens: torch.Tensor, cu_seqlens: torch
                     req_expert: Optional[torch.Tensor], max_seqlen: int, logits_mode: int = LOGITS_ALL,
                     logits: Optional[torch.Tensor] = None, hidden_in: Optional[torch.Tensor] = None,
                     hidden_out: Optional[torch.Tensor] = None, layer_begin: int = 0, layer_end: Optional[int] = None,
-                    stream=None) -> Optional[torch.Tensor]:
-    """moin_decoder_forward.  Returns logits (bf16) or None for LOGITS_NONE."""
+                    stream=None, token_expert: Optional[torch.Tensor] = None) -> Optional[torch.Tensor]:
+    """moin_decoder_forward, or moin_decoder_forward_per_token when ``token_expert`` ([T] int32) is given.
+    Returns logits (bf16) or None for LOGITS_NONE."""
     R, T = cu_seqlens.shape[0] - 1, tokens.shape[0]
     cfg = model.cfg
     if logits is None and logits_mode != LOGITS_NONE:
@@ -503,6 +504,12 @@ def decoder_forward(model: DecoderModel, tokens: torch.Tensor, cu_seqlens: torch
         logits = torch.empty(rows, cfg.vocab, dtype=torch.bfloat16, device=tokens.device)
     taps = _Taps(_ptr(hidden_in), _ptr(hidden_out), layer_begin, cfg.n_layers if layer_end is None else layer_end)
     ws = model.workspace(R, T)
+    if token_expert is not None:
+        _check(lib().moin_decoder_forward_per_token(ctypes.byref(model.c), _ptr(tokens), _ptr(cu_seqlens),
+                                                    _ptr(token_expert), R, T, max_seqlen, _ptr(logits), logits_mode,
+                                                    ctypes.byref(taps), _ptr(ws), ws.numel(), _stream(stream)),
+               "moin_decoder_forward_per_token")
+        return logits
     _check(lib().moin_decoder_forward(ctypes.byref(model.c), _ptr(tokens), _ptr(cu_seqlens), _ptr(req_expert), R, T,
                                       max_seqlen, _ptr(logits), logits_mode, ctypes.byref(taps), _ptr(ws), ws.numel(),
                                       _stream(stream)), "moin_decoder_forward")

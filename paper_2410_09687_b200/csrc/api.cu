@@ -10,7 +10,7 @@ __device__ DeviceStatus g_device_status;
 
 static thread_local int t_last_cuda_error = 0;
 static HostState g_states[kMaxDevices];
-static int g_opt_gemm_impl = 0, g_opt_stream_impl = 0;   // moin_set_option: process-wide
+static int g_opt_gemm_impl = 0;   // moin_set_option: process-wide
 
 moin_status record_cuda(cudaError_t e) {
   if (e == cudaSuccess) return MOIN_OK;
@@ -45,7 +45,6 @@ moin_status host_state(HostState** out) {
     g_state.device = dev;
   }
   g_state.gemm_impl = g_opt_gemm_impl;
-  g_state.stream_impl = g_opt_stream_impl;
   *out = &g_state;
   return MOIN_OK;
 }
@@ -101,10 +100,6 @@ int32_t moin_last_cuda_error(void) { return t_last_cuda_error; }
 moin_status moin_set_option(int32_t key, int32_t value) {
   if (key == MOIN_OPT_GEMM_IMPL && value >= 0 && value <= 2) {
     g_opt_gemm_impl = value;
-    return MOIN_OK;
-  }
-  if (key == MOIN_OPT_STREAM_IMPL && value >= 0 && value <= 3) {
-    g_opt_stream_impl = value;
     return MOIN_OK;
   }
   return MOIN_ERR_INVALID_ARG;
@@ -169,8 +164,7 @@ moin_status moin_profile_read(moin_profile_record* out, int32_t capacity, int32_
 const char* moin_kernel_name(int32_t k) {
   static const char* names[MOIN_K_COUNT] = {"route_simple", "route_tc", "route_finish", "plan", "gemm_warp", "gemm_tc",
                                             "lora_shrink_stream", "lora_expand_stream", "lora_shrink_tc",
-                                            "lora_fused_tc", "decoder_glue", "attention", "route_cluster", "kmeans_update",
-                                            "lora_fused_stream"};
+                                            "lora_fused_tc", "decoder_glue", "attention", "route_cluster", "kmeans_update"};
   return (k >= 0 && k < MOIN_K_COUNT) ? names[k] : "unknown";
 }
 
@@ -447,8 +441,8 @@ moin_status moin_plan_read(const moin_plan* plan, int32_t* n_segments, int32_t* 
 size_t moin_lora_linear_workspace_bytes(int32_t T, int32_t d_in, int32_t d_out, int32_t r) {
   if (T <= 0) return 256;
   const size_t Tp = align_up((size_t)T, kTileRows) + kTileRows;
-  const size_t parts = (size_t)lora_stream_parts(d_in > 0 ? d_in : 64);
-  size_t seg = align_up(parts * (size_t)T * (size_t)(r > 0 ? r : 8) * sizeof(float), 256) +
+  (void)d_in;
+  size_t seg = align_up((size_t)T * (size_t)(r > 0 ? r : 8) * sizeof(float), 256) +
                align_up((size_t)T * (size_t)d_out * sizeof(float), 256);
   size_t tiles = align_up(2 * Tp * (size_t)(r > 64 ? r : 64) * sizeof(__nv_bfloat16), 256);   // hi and lo parts of s * (x A^T)
   return (seg > tiles ? seg : tiles) + 256;
@@ -558,66 +552,9 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
   // projections of the group in ONE launch, so their launch and ramp-up costs are paid once per group.
   float* h[kMaxStreamJobs];
   float* y0[kMaxStreamJobs];
-  int parts[kMaxStreamJobs];
-  bool tma_stream = hs->stream_impl == 2;   // MOIN_OPT_STREAM_IMPL: TMA-staged kernels
-  for (int j = 0; j < n_jobs; ++j) tma_stream = tma_stream && lora_shrink_tma_supported(d_in[j]) && r[j] <= 64;
-  int* queue = reinterpret_cast<int*>(ws_job[0] + moin_lora_linear_workspace_bytes(T, d_in[0], d_out[0], r[0]) - 256);
-  const moin_pool* pools[kMaxStreamJobs];
-  const __nv_bfloat16* xs[kMaxStreamJobs];
-  __nv_bfloat16* ys[kMaxStreamJobs];
   for (int j = 0; j < n_jobs; ++j) {
-    pools[j] = jobs[j].pool;
-    xs[j] = (const __nv_bfloat16*)jobs[j].x;
-    ys[j] = (__nv_bfloat16*)jobs[j].y;
-    parts[j] = tma_stream ? lora_stream_parts(d_in[j]) : 1;
-    h[j] = reinterpret_cast<float*>(ws_job[j]);   // [parts][T][r] (partial) shrink results
-    y0[j] = reinterpret_cast<float*>(ws_job[j] + align_up((size_t)lora_stream_parts(d_in[j]) * (size_t)T * (size_t)r[j] * sizeof(float), 256));
-  }
-  if (!tma_stream && hs->stream_impl != 1) {
-    // One stream, programmatic dependent launches: the base GEMMs first (projections with the same d_in share a
-    // launch), then ONE launch that holds the shrink items and the expand CTAs of the whole group.  The fused
-    // launch starts beside the GEMMs (its shrink items do not depend on them); its expand CTAs wait for them.
-    {
-      ProfScope prof(MOIN_K_GEMM_TC, 1, s);
-      for (int j0 = 0; j0 < n_jobs;) {
-        if (!use_tc[j0]) {
-          if ((st = record_cuda(launch_gemm_warp(xs[j0], (const __nv_bfloat16*)jobs[j0].W, ys[j0], y0[j0], T, d_in[j0],
-                                                 d_out[j0], s))))
-            return st;
-          ++j0;
-          continue;
-        }
-        const __nv_bfloat16* gw[kTcMaxStoreJobs];
-        int gd[kTcMaxStoreJobs], n = 0;
-        while (j0 + n < n_jobs && n < kTcMaxStoreJobs && use_tc[j0 + n] && d_in[j0 + n] == d_in[j0]) {
-          gw[n] = (const __nv_bfloat16*)jobs[j0 + n].W;
-          gd[n] = d_out[j0 + n];
-          ++n;
-        }
-        if ((st = launch_tc_gemm_group(hs, xs + j0, gw, ys + j0, y0 + j0, gd, n, T, d_in[j0], s))) return st;
-        j0 += n;
-      }
-    }
-    ShrinkJobs sj = {};
-    ExpandJobs ej = {};
-    sj.n = ej.n = n_jobs;
-    for (int j = 0; j < n_jobs; ++j) {
-      sj.x[j] = xs[j];
-      sj.A[j] = (const __nv_bfloat16*)jobs[j].pool->A;
-      sj.h[j] = h[j];
-      sj.slot_of_expert[j] = jobs[j].pool->slot_of_expert;
-      sj.r[j] = r[j];
-      sj.d_in[j] = d_in[j];
-      ej.h[j] = h[j];
-      ej.B[j] = (const __nv_bfloat16*)jobs[j].pool->B;
-      ej.y0[j] = y0[j];
-      ej.y[j] = ys[j];
-      ej.slot_of_expert[j] = jobs[j].pool->slot_of_expert;
-      ej.r[j] = r[j];
-      ej.d_out[j] = d_out[j];
-    }
-    ProfScope prof(MOIN_K_FUSED_STREAM, 1, s);
-    return record_cuda(launch_lora_fused_stream(pv, sj, ej, scale, hs->n_sms, hs->status, s));
+    h[j] = reinterpret_cast<float*>(ws_job[j]);   // [T][r] shrink results
+    y0[j] = reinterpret_cast<float*>(ws_job[j] + align_up((size_t)T * (size_t)r[j] * sizeof(float), 256));
   }
   cudaError_t ce = cudaEventRecord(hs->ev_fork, s);
   if (ce != cudaSuccess) return record_cuda(ce);
@@ -627,9 +564,9 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
     if (ce != cudaSuccess) return record_cuda(ce);
     ProfScope prof(use_tc[j] ? MOIN_K_GEMM_TC : MOIN_K_GEMM_WARP, 1, hs->side[j]);
     moin_status sj;
-    if (use_tc[j])
+    if (use_tc[j])   // the group's base GEMMs together get three quarters of the SMs, the shrink beside them the rest
       sj = launch_tc_gemm(hs, (const __nv_bfloat16*)jobs[j].x, (const __nv_bfloat16*)jobs[j].W, (__nv_bfloat16*)jobs[j].y,
-                          y0[j], T, d_in[j], d_out[j], hs->side[j]);
+                          y0[j], T, d_in[j], d_out[j], hs->side[j], hs->n_sms * 3 / 4 / n_jobs);
     else
       sj = record_cuda(launch_gemm_warp((const __nv_bfloat16*)jobs[j].x, (const __nv_bfloat16*)jobs[j].W,
                                         (__nv_bfloat16*)jobs[j].y, y0[j], T, d_in[j], d_out[j], hs->side[j]));
@@ -638,21 +575,17 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
   moin_status st_shrink;
   {
     ProfScope prof(MOIN_K_SHRINK_STREAM, 1, s);
-    if (tma_stream) {
-      st_shrink = launch_lora_shrink_tma(hs, pv, pools, xs, h, n_jobs, queue, lora_stream_ring_bytes(), s);
-    } else {
-      ShrinkJobs sj = {};
-      sj.n = n_jobs;
-      for (int j = 0; j < n_jobs; ++j) {
-        sj.x[j] = (const __nv_bfloat16*)jobs[j].x;
-        sj.A[j] = (const __nv_bfloat16*)jobs[j].pool->A;
-        sj.h[j] = h[j];
-        sj.slot_of_expert[j] = jobs[j].pool->slot_of_expert;
-        sj.r[j] = r[j];
-        sj.d_in[j] = d_in[j];
-      }
-      st_shrink = record_cuda(launch_lora_shrink_stream(pv, sj, hs->n_sms, s));
+    ShrinkJobs sj = {};
+    sj.n = n_jobs;
+    for (int j = 0; j < n_jobs; ++j) {
+      sj.x[j] = (const __nv_bfloat16*)jobs[j].x;
+      sj.A[j] = (const __nv_bfloat16*)jobs[j].pool->A;
+      sj.h[j] = h[j];
+      sj.slot_of_expert[j] = jobs[j].pool->slot_of_expert;
+      sj.r[j] = r[j];
+      sj.d_in[j] = d_in[j];
     }
+    st_shrink = record_cuda(launch_lora_shrink_stream(pv, sj, hs->n_sms, s));
   }
   // always join, even after a failed launch, so the side streams never outlive the call's ordering
   for (int j = 0; j < n_jobs; ++j) {
@@ -663,8 +596,6 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
   if (st_gemm) return st_gemm;
   if (st_shrink) return st_shrink;
   ProfScope prof(MOIN_K_EXPAND_STREAM, 1, s);
-  if (tma_stream)
-    return launch_lora_expand_tma(hs, pv, pools, h, parts, y0, ys, n_jobs, scale, queue, lora_stream_ring_bytes(), s);
   ExpandJobs ej = {};
   ej.n = n_jobs;
   for (int j = 0; j < n_jobs; ++j) {

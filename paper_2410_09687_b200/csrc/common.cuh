@@ -24,9 +24,6 @@ constexpr int kPlanHeaderWords = 16;
 enum PlanHeader { PH_NSEG = 0, PH_NTILES = 1, PH_NLORA = 2, PH_MAXSEG = 3, PH_T = 4, PH_E = 5 };
 constexpr int kPlanChunk = 256;   // tokens per histogram chunk
 constexpr int kTileRows = 128;    // rows per GEMM tile
-constexpr int kSyncHeaderWords = 16;   // plan sync area: [SY_DONE] CTAs finished, then one counter per (job, segment)
-constexpr int kPlanSyncJobs = 4;       // = kMaxStreamJobs
-enum PlanSync { SY_DONE = 0 };
 
 struct PlanView {   // pointers into the plan buffer
   int* header;
@@ -41,8 +38,6 @@ struct PlanView {   // pointers into the plan buffer
   int* key;          // [T]   scratch
   int* keybase;      // [E+1] scratch
   int* hist;         // [n_chunks * (E+1)] scratch
-  int* sync;         // [kSyncHeaderWords + kMaxStreamJobs * (Smax + 1)] counters of the fused short-segment launch:
-                     // zero after the plan build and again after every launch that used them
   int T, E, Smax, n_chunks;
 };
 
@@ -68,7 +63,6 @@ inline PlanView plan_view(void* buffer, int T, int E, size_t* total_words = null
   v.key = take(T);
   v.keybase = take(E + 2);
   v.hist = take((size_t)v.n_chunks * (size_t)(E + 1));
-  v.sync = take(kSyncHeaderWords + (size_t)kPlanSyncJobs * (size_t)(v.Smax + 1));
   if (total_words) *total_words = off;
   return v;
 }
@@ -119,7 +113,6 @@ cudaError_t launch_plan_build(const int* token_expert, const PlanView& v, Device
                               cudaStream_t stream);
 // Register-fed short-segment kernels: one launch covers up to kMaxStreamJobs projections sharing a plan.
 constexpr int kMaxStreamJobs = 4;
-static_assert(kMaxStreamJobs == kPlanSyncJobs, "plan sync area");
 struct ShrinkJobs {
   const __nv_bfloat16* x[kMaxStreamJobs];
   const __nv_bfloat16* A[kMaxStreamJobs];
@@ -135,14 +128,11 @@ struct ExpandJobs {
   __nv_bfloat16* y[kMaxStreamJobs];
   const int* slot_of_expert[kMaxStreamJobs];
   int r[kMaxStreamJobs], d_out[kMaxStreamJobs], rows_per_item[kMaxStreamJobs], per_seg[kMaxStreamJobs];
-  int need[kMaxStreamJobs];   // fused launch: shrink items per segment that must have signalled before the expand reads h
   int n;
 };
 cudaError_t launch_lora_shrink_stream(const PlanView& pv, ShrinkJobs jobs, int n_sms, cudaStream_t stream);
 cudaError_t launch_lora_expand_stream(const PlanView& pv, ExpandJobs jobs, float scale, int n_sms,
                                       cudaStream_t stream);
-cudaError_t launch_lora_fused_stream(const PlanView& pv, ShrinkJobs sj, ExpandJobs ej, float scale, int n_sms,
-                                     DeviceStatus* status, cudaStream_t stream);
 cudaError_t launch_gemm_warp(const __nv_bfloat16* x, const __nv_bfloat16* W, __nv_bfloat16* y, float* y0, int T,
                              int d_in, int d_out, cudaStream_t stream);
 cudaError_t launch_route_top2_simple(const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
@@ -175,7 +165,6 @@ struct HostState {
   int device = -1;
   int n_sms = 0;
   int gemm_impl = 0;               // MOIN_OPT_GEMM_IMPL (process-wide option, copied in on every call)
-  int stream_impl = 0;             // MOIN_OPT_STREAM_IMPL
   // fork/join inside one call: independent kernels of a call run on `side` between two events
   cudaStream_t side[kMaxStreamJobs] = {nullptr, nullptr, nullptr, nullptr};
   cudaEvent_t ev_fork = nullptr, ev_join[kMaxStreamJobs] = {nullptr, nullptr, nullptr, nullptr};
@@ -188,9 +177,7 @@ moin_status record_cuda(cudaError_t e);       // MOIN_OK or MOIN_ERR_CUDA (remem
 // that attribute per device, so the "already done" note is kept per device too (slot = one id per kernel).
 enum {
   OPTIN_TC_GEMM = 0,        // + 4 * (BN index) + EPI, 12 entries; + 12 for the short-ring instantiations
-  OPTIN_ROUTE_CLUSTER = 24, OPTIN_ROUTE_SIMPLE = 25, OPTIN_SHRINK_TMA = 26, OPTIN_EXPAND_TMA = 27,
-  OPTIN_LORA_FUSED = 28, OPTIN_ATTENTION = 29, OPTIN_ROUTE_PLAN = 30,
-  OPTIN_TC_GROUP = 31       // + BN index, 3 entries
+  OPTIN_ROUTE_CLUSTER = 24, OPTIN_ROUTE_SIMPLE = 25, OPTIN_ATTENTION = 29
 };
 template <class Fn>
 inline cudaError_t ensure_smem_optin(int slot, Fn* fn, size_t bytes) {

@@ -4,9 +4,11 @@
 
 namespace moin {
 
-// token -> (position inside its request, expert of its request).  One CTA per request.
+// token -> (position inside its request, its expert: the caller's per-token id if given, else the expert of its
+// request).  One CTA per request.
 __global__ void __launch_bounds__(256)
-token_meta_kernel(const int* __restrict__ cu, const int* __restrict__ req_expert, int R, int* __restrict__ pos,
+token_meta_kernel(const int* __restrict__ cu, const int* __restrict__ req_expert,
+                  const int* __restrict__ token_expert_in, int R, int* __restrict__ pos,
                   int* __restrict__ token_expert, int* __restrict__ last_row) {
   const int r = blockIdx.x;
   if (r >= R) return;
@@ -14,7 +16,7 @@ token_meta_kernel(const int* __restrict__ cu, const int* __restrict__ req_expert
   const int e = req_expert ? req_expert[r] : -1;
   for (int t = t0 + threadIdx.x; t < t1; t += blockDim.x) {
     pos[t] = t - t0;
-    token_expert[t] = e;
+    token_expert[t] = token_expert_in ? token_expert_in[t] : e;
   }
   if (threadIdx.x == 0) last_row[r] = (t1 > t0) ? t1 - 1 : -1;
 }
@@ -343,10 +345,11 @@ extern "C" size_t moin_decoder_workspace_bytes(const moin_model* model, int32_t 
   return carve(model, R, T, T, nullptr).total + 256;
 }
 
-extern "C" moin_status moin_decoder_forward(const moin_model* m, const int32_t* tokens, const int32_t* cu_seqlens,
-                                            const int32_t* req_expert, int32_t R, int32_t T, int32_t max_seqlen,
-                                            void* logits, int32_t logits_mode, const moin_decoder_taps* taps,
-                                            void* workspace, size_t workspace_bytes, moin_stream stream) {
+static moin_status decoder_forward_impl(const moin_model* m, const int32_t* tokens, const int32_t* cu_seqlens,
+                                        const int32_t* req_expert, const int32_t* token_expert_in, int32_t R,
+                                        int32_t T, int32_t max_seqlen, void* logits, int32_t logits_mode,
+                                        const moin_decoder_taps* taps, void* workspace, size_t workspace_bytes,
+                                        moin_stream stream) {
   if (!m || R < 0 || T < 0) return MOIN_ERR_INVALID_ARG;
   if (R == 0 || T == 0) return MOIN_OK;
   if (!cu_seqlens || !m->W || !m->attn_norm || !m->mlp_norm || !m->final_norm) return MOIN_ERR_INVALID_ARG;
@@ -370,14 +373,16 @@ extern "C" moin_status moin_decoder_forward(const moin_model* m, const int32_t* 
   const int qd = nh * 64, kvd = nkv * 64;
 
   { ProfScope prof(MOIN_K_GLUE, 2, s);
-  token_meta_kernel<<<R, 256, 0, s>>>(cu_seqlens, req_expert, R, w.pos, w.token_expert, w.last_row);
+  token_meta_kernel<<<R, 256, 0, s>>>(cu_seqlens, req_expert, token_expert_in, R, w.pos, w.token_expert, w.last_row);
   rope_table_kernel<<<(max_seqlen * 32 + 255) / 256, 256, 0, s>>>(w.rope, max_seqlen, 32, (double)m->rope_base); }
   moin_plan plan;
   memset(&plan, 0, sizeof(plan));
-  const bool lora = m->pools != nullptr && req_expert != nullptr;
+  const bool lora = m->pools != nullptr && (req_expert != nullptr || token_expert_in != nullptr);
   if (lora) {
     plan.buffer = w.plan; plan.buffer_bytes = w.plan_bytes; plan.T = T; plan.E = m->E;
-    plan.mode = (T / R >= 64) ? MOIN_PLAN_TILES : MOIN_PLAN_SEGMENTS;
+    // one expert per request: the run lengths are the request lengths; one per token: they depend on the ids, so
+    // the plan decides after it has grouped them (reads its header back: one synchronisation of the stream)
+    plan.mode = token_expert_in ? MOIN_PLAN_AUTO : ((T / R >= 64) ? MOIN_PLAN_TILES : MOIN_PLAN_SEGMENTS);
     st = moin_plan_build(w.token_expert, &plan, stream);
     if (st) return st;
   }
@@ -456,4 +461,22 @@ extern "C" moin_status moin_decoder_forward(const moin_model* m, const int32_t* 
     if (st) return st;
   }
   return record_cuda(cudaGetLastError());
+}
+
+extern "C" moin_status moin_decoder_forward(const moin_model* m, const int32_t* tokens, const int32_t* cu_seqlens,
+                                            const int32_t* req_expert, int32_t R, int32_t T, int32_t max_seqlen,
+                                            void* logits, int32_t logits_mode, const moin_decoder_taps* taps,
+                                            void* workspace, size_t workspace_bytes, moin_stream stream) {
+  return decoder_forward_impl(m, tokens, cu_seqlens, req_expert, nullptr, R, T, max_seqlen, logits, logits_mode, taps,
+                              workspace, workspace_bytes, stream);
+}
+
+extern "C" moin_status moin_decoder_forward_per_token(const moin_model* m, const int32_t* tokens,
+                                                      const int32_t* cu_seqlens, const int32_t* token_expert, int32_t R,
+                                                      int32_t T, int32_t max_seqlen, void* logits, int32_t logits_mode,
+                                                      const moin_decoder_taps* taps, void* workspace,
+                                                      size_t workspace_bytes, moin_stream stream) {
+  if (!token_expert) return MOIN_ERR_INVALID_ARG;
+  return decoder_forward_impl(m, tokens, cu_seqlens, nullptr, token_expert, R, T, max_seqlen, logits, logits_mode, taps,
+                              workspace, workspace_bytes, stream);
 }

@@ -32,41 +32,6 @@ __device__ __forceinline__ V pick(const V (&arr)[kMaxStreamJobs], int j) {
   return v;
 }
 
-// Programmatic dependent launch: wait for the grid this one was launched behind (no-op without one), and allow
-// the grid launched behind this one to start.
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
-template <bool COHERENT>
-__device__ __forceinline__ float ld_base(const float* p) { return COHERENT ? __ldcg(p) : __ldg(p); }
-
-// Warp-wide bounded wait until *flag >= need: lane 0 polls (acquire), the warp then synchronises, which orders
-// the other lanes' later reads behind it.  On expiry: status flag, false for the whole warp.
-__device__ __forceinline__ bool wait_ready(const int* flag, int need, DeviceStatus* status) {
-  int ok = 1;
-  if ((threadIdx.x & 31) == 0) {
-    int v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-    unsigned long long t0 = 0;
-    for (uint32_t spins = 1; v < need; ++spins) {
-      __nanosleep(64);
-      asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-      if ((spins & 0xFFu) == 0 && v < need) {
-        unsigned long long now;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
-        if (t0 == 0) t0 = now;
-        if (now - t0 > 2000000000ull) {
-          atomicExch(&status->timeout_flag, 1);
-          atomicExch(&status->timeout_site, 21);
-          ok = 0;
-          break;
-        }
-      }
-    }
-  }
-  return __shfl_sync(0xffffffffu, ok, 0) != 0;
-}
-
 struct ItemRef { int job, seg, sub; };
 template <class Jobs>
 __device__ __forceinline__ ItemRef decode_item(int item, int nseg, const Jobs& jobs) {
@@ -108,12 +73,23 @@ __device__ __forceinline__ SegMeta load_seg(const int4* __restrict__ seg_tab, co
 // the hardware's block scheduler hands the items out as slots free up, so a launch ends evenly whatever
 // the base GEMMs on the side streams occupy, and a CTA's metadata hops (segment count, table entry,
 // slot) hide behind the streams of the other CTAs on its SM.
-// One shrink work item: 16 adapter rows of one (job, segment), all the segment's tokens.
-__device__ __forceinline__ void shrink_item(const SegMeta& cur, const int* __restrict__ perm, const ShrinkJobs& jobs,
-                                            float (&red)[kShrinkWarps][32][4]) {
+__global__ void __launch_bounds__(kShrinkThreads, 6)
+lora_shrink_stream_kernel(const int* __restrict__ header, const int* __restrict__ perm,
+                          const int4* __restrict__ seg_tab, const ShrinkJobs jobs) {
+  __shared__ float red[kShrinkWarps][32][4];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  {
+  const int nseg = header[PH_NSEG];
+  int items = 0;
+#pragma unroll
+  for (int j = 0; j < kMaxStreamJobs; ++j)
+    if (j < jobs.n) items += nseg * jobs.per_seg[j];
+  int item = blockIdx.x;
+  SegMeta nxt = load_seg(seg_tab, jobs, item, items, nseg);
+  for (; item < items; item += gridDim.x) {
+    const SegMeta cur = nxt;
+    nxt = load_seg(seg_tab, jobs, item + gridDim.x, items, nseg);  // lookahead
+    if (cur.slot < 0) continue;  // uniform per CTA
     const int r = pick(jobs.r, cur.job), d_in = pick(jobs.d_in, cur.job);
     const __nv_bfloat16* __restrict__ x = pick(jobs.x, cur.job);
     const __nv_bfloat16* __restrict__ A = pick(jobs.A, cur.job);
@@ -180,25 +156,6 @@ __device__ __forceinline__ void shrink_item(const SegMeta& cur, const int* __res
   }
 }
 
-__global__ void __launch_bounds__(kShrinkThreads, 6)
-lora_shrink_stream_kernel(const int* __restrict__ header, const int* __restrict__ perm,
-                          const int4* __restrict__ seg_tab, const ShrinkJobs jobs) {
-  __shared__ float red[kShrinkWarps][32][4];
-  const int nseg = header[PH_NSEG];
-  int items = 0;
-#pragma unroll
-  for (int j = 0; j < kMaxStreamJobs; ++j)
-    if (j < jobs.n) items += nseg * jobs.per_seg[j];
-  int item = blockIdx.x;
-  SegMeta nxt = load_seg(seg_tab, jobs, item, items, nseg);
-  for (; item < items; item += gridDim.x) {
-    const SegMeta cur = nxt;
-    nxt = load_seg(seg_tab, jobs, item + gridDim.x, items, nseg);  // lookahead
-    if (cur.slot < 0) continue;  // uniform per CTA
-    shrink_item(cur, perm, jobs, red);
-  }
-}
-
 // y[perm[pos]][j] = bf16( y0[perm[pos]][j] + scale * sum_rho B[slot][j][rho] * h[pos][rho] )
 // h is split into bf16 hi + lo parts (two MMAs) so the low-rank term keeps ~fp32 accuracy.
 //
@@ -208,20 +165,15 @@ lora_shrink_stream_kernel(const int* __restrict__ header, const int* __restrict_
 // of adapter bytes, whatever the mix of projection widths in the launch, and a warp's range is contiguous
 // in memory inside a (segment, job).  A warp walks its range kExpandTilesPerBatch tiles at a time with
 // the adapter rows and the base values y0 of a batch loaded together.  `jobs.per_seg[j]` = tiles of job j.
-//
-// FUSED (the expand part of lora_fused_stream_kernel): the shrink items of the same launch produce h, so a
-// (segment, job) piece first waits until all of that pair's shrink items have signalled `ready`, h and y0 are
-// read through L2 (never through the read-only path), and the warp waits once for the preceding base-GEMM
-// launch (programmatic dependent launch) before it touches y0 or y.  Returns false if a wait ran out.
-template <int P, bool FUSED>  // P: number of 32-wide rho groups, ceil(max r / 32)
-__device__ __forceinline__ bool expand_range(long long wid, long long nw, const int* __restrict__ header,
-                                             const int* __restrict__ perm, const int4* __restrict__ seg_tab,
-                                             const ExpandJobs& jobs, float scale, int tps, const int* ready,
-                                             int ready_pitch, DeviceStatus* status) {
+template <int P>  // number of 32-wide rho groups: ceil(max r / 32)
+__global__ void __launch_bounds__(kExpandThreads, 4)
+lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict__ perm,
+                          const int4* __restrict__ seg_tab, const ExpandJobs jobs, float scale, int tps) {
   constexpr int TB = P > 2 ? 1 : kExpandTilesPerBatch;   // wide ranks: one tile's rows already fill the load registers
-  const int lane = threadIdx.x & 31;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  if (FUSED) grid_dependency_wait();
+  const long long wid = (long long)blockIdx.x * (kExpandThreads / 32) + warp;
+  const long long nw = (long long)gridDim.x * (kExpandThreads / 32);
   const int nseg = __ldg(header + PH_NSEG);
   const long long units = (long long)nseg * tps;
   long long u = units * wid / nw;
@@ -254,9 +206,8 @@ __device__ __forceinline__ bool expand_range(long long wid, long long nw, const 
       const int slot = pick(slots, job);
       if (slot >= 0) {
         const int r = pick(jobs.r, job), d_out = pick(jobs.d_out, job);
-        if (FUSED && !wait_ready(ready + (size_t)job * ready_pitch + seg, pick(jobs.need, job), status)) return false;
-        const float* h = pick(jobs.h, job);
-        const float* y0 = pick(jobs.y0, job);
+        const float* __restrict__ h = pick(jobs.h, job);
+        const float* __restrict__ y0 = pick(jobs.y0, job);
         __nv_bfloat16* __restrict__ y = pick(jobs.y, job);
         const __nv_bfloat16* Bs = pick(jobs.B, job) + (size_t)slot * (size_t)d_out * (size_t)r;
         for (int tc = 0; tc < n; tc += 8) {
@@ -269,9 +220,8 @@ __device__ __forceinline__ bool expand_range(long long wid, long long nw, const 
             const int rb = 32 * p + 8 * t;
             float v[8];
             if (vx && rb < r) {
-              const float4* hp = reinterpret_cast<const float4*>(h + (size_t)(s0 + tc + g) * r + rb);
-              const float4 f0 = FUSED ? __ldcg(hp) : *hp;
-              const float4 f1 = FUSED ? __ldcg(hp + 1) : *(hp + 1);
+              const float4 f0 = *reinterpret_cast<const float4*>(h + (size_t)(s0 + tc + g) * r + rb);
+              const float4 f1 = *reinterpret_cast<const float4*>(h + (size_t)(s0 + tc + g) * r + rb + 4);
               v[0] = f0.x; v[1] = f0.y; v[2] = f0.z; v[3] = f0.w; v[4] = f1.x; v[5] = f1.y; v[6] = f1.z; v[7] = f1.w;
             } else {
 #pragma unroll
@@ -301,10 +251,10 @@ __device__ __forceinline__ bool expand_range(long long wid, long long nw, const 
                 a0[i][p] = (va && rb < r) ? ldg_stream(Bs + (size_t)ja * r + rb) : z;
                 a1[i][p] = (vc && rb < r) ? ldg_stream(Bs + (size_t)jc * r + rb) : z;
               }
-              b0[i][0] = (va && row_c0 >= 0) ? ld_base<FUSED>(y0 + (size_t)row_c0 * d_out + ja) : 0.f;
-              b0[i][1] = (va && row_c1 >= 0) ? ld_base<FUSED>(y0 + (size_t)row_c1 * d_out + ja) : 0.f;
-              b0[i][2] = (vc && row_c0 >= 0) ? ld_base<FUSED>(y0 + (size_t)row_c0 * d_out + jc) : 0.f;
-              b0[i][3] = (vc && row_c1 >= 0) ? ld_base<FUSED>(y0 + (size_t)row_c1 * d_out + jc) : 0.f;
+              b0[i][0] = (va && row_c0 >= 0) ? __ldg(y0 + (size_t)row_c0 * d_out + ja) : 0.f;
+              b0[i][1] = (va && row_c1 >= 0) ? __ldg(y0 + (size_t)row_c1 * d_out + ja) : 0.f;
+              b0[i][2] = (vc && row_c0 >= 0) ? __ldg(y0 + (size_t)row_c0 * d_out + jc) : 0.f;
+              b0[i][3] = (vc && row_c1 >= 0) ? __ldg(y0 + (size_t)row_c1 * d_out + jc) : 0.f;
             }
 #pragma unroll
             for (int i = 0; i < TB; ++i) {
@@ -337,81 +287,6 @@ __device__ __forceinline__ bool expand_range(long long wid, long long nw, const 
       rem = 0;
       ++job;
     }
-  }
-  return true;
-}
-
-template <int P>
-__global__ void __launch_bounds__(kExpandThreads, 4)
-lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict__ perm,
-                          const int4* __restrict__ seg_tab, const ExpandJobs jobs, float scale, int tps) {
-  const long long wid = (long long)blockIdx.x * (kExpandThreads / 32) + (threadIdx.x >> 5);
-  const long long nw = (long long)gridDim.x * (kExpandThreads / 32);
-  expand_range<P, false>(wid, nw, header, perm, seg_tab, jobs, scale, tps, nullptr, 0, nullptr);
-}
-
-// Shrink and expand of a group in ONE launch.  The first `n_shrink` CTAs are the shrink items, ordered
-// (segment, job, 16-row block); the rest are the expand CTAs, whose warps take equal ranges of output tiles
-// ordered (segment, job, tile).  There is no grid-wide barrier between the two: a shrink CTA bumps the
-// `ready` counter of its (job, segment) once its rows of h are written, and an expand warp waits for exactly
-// the pairs it is about to use, so adapter bytes of B start streaming while other segments' A rows are still
-// in flight.  Shrink CTAs come first in launch order and never wait, so every wait ends; waits are bounded all
-// the same (status flag, clean return).  The last CTA to finish clears the counters for the next launch that
-// uses the plan.  With programmatic dependent launch the whole grid may start while the preceding base GEMM
-// is still running: shrink CTAs do not depend on it, expand warps wait for it before reading y0.
-template <int P>
-__global__ void __launch_bounds__(kExpandThreads, 4)
-lora_fused_stream_kernel(const int* __restrict__ header, const int* __restrict__ perm,
-                         const int4* __restrict__ seg_tab, const ShrinkJobs sj, const ExpandJobs ej, float scale,
-                         int tps, int n_shrink, int shrink_per_seg, int* sync, int ready_pitch, DeviceStatus* status) {
-  static_assert(kShrinkThreads == kExpandThreads, "one block shape for both roles");
-  __shared__ float red[kShrinkWarps][32][4];
-  grid_launch_dependents();
-  int* ready = sync + kSyncHeaderWords;
-  if ((int)blockIdx.x < n_shrink) {
-    const int nseg = header[PH_NSEG];
-    const int seg = blockIdx.x / shrink_per_seg;
-    if (seg < nseg) {
-      int rem = blockIdx.x - seg * shrink_per_seg, job = 0;
-#pragma unroll
-      for (int j = 0; j + 1 < kMaxStreamJobs; ++j) {
-        if (job == j && j + 1 < sj.n && rem >= sj.per_seg[j]) {
-          rem -= sj.per_seg[j];
-          job = j + 1;
-        }
-      }
-      const int4 e = __ldg(seg_tab + seg);   // (expert, start, length, -)
-      SegMeta cur;
-      cur.slot = __ldg(pick(sj.slot_of_expert, job) + e.x);
-      cur.s0 = e.y; cur.n = e.z; cur.job = job; cur.sub = rem;
-      if (cur.slot >= 0) {
-        shrink_item(cur, perm, sj, red);
-        // h rows of this item are written by warp 0: make them visible, then count the item in
-        __syncthreads();
-        if (threadIdx.x == 0) {
-          __threadfence();
-          atomicAdd(ready + (size_t)job * ready_pitch + seg, 1);
-        }
-      }
-    }
-  } else {
-    const long long wid = (long long)((int)blockIdx.x - n_shrink) * (kExpandThreads / 32) + (threadIdx.x >> 5);
-    const long long nw = (long long)((int)gridDim.x - n_shrink) * (kExpandThreads / 32);
-    expand_range<P, true>(wid, nw, header, perm, seg_tab, ej, scale, tps, ready, ready_pitch, status);
-  }
-  // the last CTA out leaves the counters at zero for the next launch on this plan
-  __syncthreads();
-  __shared__ int s_last;
-  if (threadIdx.x == 0) {
-    __threadfence();
-    s_last = (atomicAdd(sync + SY_DONE, 1) == (int)gridDim.x - 1);
-  }
-  __syncthreads();
-  if (s_last) {
-    __threadfence();
-    const int n = kMaxStreamJobs * ready_pitch;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) ready[i] = 0;
-    if (threadIdx.x == 0) sync[SY_DONE] = 0;
   }
 }
 
@@ -451,46 +326,6 @@ cudaError_t launch_lora_expand_stream(const PlanView& pv, ExpandJobs jobs, float
   else
     lora_expand_stream_kernel<4><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale, tps);
   return cudaGetLastError();
-}
-
-// Shrink + expand of a group in one launch (see lora_fused_stream_kernel).  `sync` = the plan's counters.
-// Launched with the programmatic-stream-serialization attribute: it may start while the kernel before it on the
-// stream (the group's base GEMM) is still running.
-cudaError_t launch_lora_fused_stream(const PlanView& pv, ShrinkJobs sj, ExpandJobs ej, float scale, int n_sms,
-                                     DeviceStatus* status, cudaStream_t stream) {
-  int shrink_per_seg = 0, tps = 0, rmax = 0;
-  for (int j = 0; j < sj.n; ++j) {
-    sj.per_seg[j] = (sj.r[j] + 15) / 16;
-    shrink_per_seg += sj.per_seg[j];
-    ej.need[j] = sj.per_seg[j];
-    ej.rows_per_item[j] = 16;
-    ej.per_seg[j] = (ej.d_out[j] + 15) / 16;
-    tps += ej.per_seg[j];
-    rmax = ej.r[j] > rmax ? ej.r[j] : rmax;
-  }
-  const long n_shrink = (long)pv.Smax * shrink_per_seg;
-  const long max_ctas = ((long)pv.Smax * tps + 2 * (kExpandThreads / 32) - 1) / (2 * (kExpandThreads / 32));
-  const int n_expand = stream_grid(max_ctas, n_sms, 4);
-  if (n_shrink + n_expand > 0x7fffffffL) return cudaErrorInvalidConfiguration;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(n_shrink + n_expand));
-  cfg.blockDim = dim3(kExpandThreads);
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  const int ns = (int)n_shrink, pitch = pv.Smax + 1;
-  if (rmax <= 32)
-    return cudaLaunchKernelEx(&cfg, lora_fused_stream_kernel<1>, (const int*)pv.header, (const int*)pv.perm,
-                              (const int4*)pv.seg_tab, sj, ej, scale, tps, ns, shrink_per_seg, pv.sync, pitch, status);
-  if (rmax <= 64)
-    return cudaLaunchKernelEx(&cfg, lora_fused_stream_kernel<2>, (const int*)pv.header, (const int*)pv.perm,
-                              (const int4*)pv.seg_tab, sj, ej, scale, tps, ns, shrink_per_seg, pv.sync, pitch, status);
-  return cudaLaunchKernelEx(&cfg, lora_fused_stream_kernel<4>, (const int*)pv.header, (const int*)pv.perm,
-                            (const int4*)pv.seg_tab, sj, ej, scale, tps, ns, shrink_per_seg, pv.sync, pitch, status);
 }
 
 }  // namespace moin

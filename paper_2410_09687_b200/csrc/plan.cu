@@ -178,7 +178,6 @@ __global__ void __launch_bounds__(1024) plan_scan_kernel(PlanView v, int do_pref
   const int tid = threadIdx.x;
   const int T = v.T, E = v.E, nc = v.n_chunks;
   const size_t pitch = (size_t)(E + 1);
-  for (int i = tid; i < kSyncHeaderWords + kPlanSyncJobs * (v.Smax + 1); i += NT) v.sync[i] = 0;
 
   // 1. per expert id: prefix over chunks (in place) and total (done by plan_prefix_kernel for multi-chunk batches)
   for (int k = tid; do_prefix && k <= E; k += 1024) {
@@ -245,7 +244,6 @@ __global__ void __launch_bounds__(NT) plan_small_kernel(const int* __restrict__ 
   __shared__ int s_carry[2];
   const int tid = threadIdx.x;
   const int T = v.T, E = v.E;
-  for (int i = tid; i < kSyncHeaderWords + kPlanSyncJobs * (v.Smax + 1); i += NT) v.sync[i] = 0;
   int k = 0x1FFFFF;  // padding sorts last
   if (tid < T) {
     int e = token_expert[tid];

@@ -28,14 +28,9 @@ namespace moin {
 
 constexpr int kBM = 128, kBK = 64;
 constexpr int kTcThreads = 192;
-enum { EPI_STORE = 0, EPI_ROUTER = 1, EPI_SHRINK = 2, EPI_ROUTER2 = 3, EPI_STORE_GROUP = 4 };   // ROUTER2: best and runner-up
-// EPI_STORE_GROUP: EPI_STORE (no plan, no tail) for up to kMaxStoreJobs projections with the same row count and
-// reduction length in ONE launch, tiles laid out job after job.  The kernel first waits for the grid it was launched
-// behind and then lets the next one start (programmatic dependent launch): the group's fused shrink/expand launch
-// streams adapters beside it.
+enum { EPI_STORE = 0, EPI_ROUTER = 1, EPI_SHRINK = 2, EPI_ROUTER2 = 3 };   // ROUTER2: best and runner-up
 
 constexpr int kMaxShrinkJobs = 3;
-constexpr int kMaxStoreJobs = 3;
 struct TcParams {
   int M, N, K;                 // problem: rows, output columns, reduction length
   // plan tiles (nullptr -> regular grid over M)
@@ -61,13 +56,6 @@ struct TcParams {
   const int* slot_tabs[3];
   __nv_bfloat16* ys[3];
   __nv_bfloat16* ys_lo[3];
-  // EPI_STORE_GROUP: job j has g_N[j] output columns, its tiles end before index g_tile_end[j], reads x / W through
-  // the j-th A-side / B-side map and writes g_y[j] (bf16) and g_y0[j] (fp32, optional), leading dimension g_N[j]
-  int g_n;
-  int g_N[3];
-  int g_tile_end[3];
-  __nv_bfloat16* g_y[3];
-  float* g_y0[3];
   const float* inv_norm;       // EPI_ROUTER
   unsigned long long* keys;    // EPI_ROUTER / EPI_ROUTER2: best (similarity, index) key per row
   unsigned long long* keys2;   // EPI_ROUTER2: runner-up key per row
@@ -140,32 +128,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  if (EPI == EPI_STORE_GROUP) {   // inputs come from the grid before; the grid behind may start beside this one
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  }
 
   const bool planned = p.header != nullptr;
   const int tiles_n = (p.N + BN - 1) / BN;
   const int tiles_m = planned ? p.header[PH_NTILES] : (p.M + kBM - 1) / kBM;
   const int n_jobs = (EPI == EPI_SHRINK && p.n_jobs > 1) ? p.n_jobs : 1;   // EPI_SHRINK: tiles_n == 1
-  const int total = (EPI == EPI_STORE_GROUP) ? p.g_tile_end[p.g_n - 1] : tiles_m * tiles_n * n_jobs;
+  const int total = tiles_m * tiles_n * n_jobs;
   const int nkb_main = (p.K + kBK - 1) / kBK;
 
-  int job = 0;   // projection of the current tile (EPI_SHRINK / EPI_STORE_GROUP with several jobs), set by tile_info
-  int cur_N = p.N;   // output columns of the current tile's projection
+  int job = 0;   // projection of the current tile (EPI_SHRINK with several jobs), set by tile_info
   auto tile_info = [&](int tile, int& row0, int& rows, int& n0, int& slot) {
-    if (EPI == EPI_STORE_GROUP) {
-      job = (p.g_n > 1 && tile >= p.g_tile_end[0]) ? ((p.g_n > 2 && tile >= p.g_tile_end[1]) ? 2 : 1) : 0;
-      const int t0 = job == 0 ? 0 : (job == 1 ? p.g_tile_end[0] : p.g_tile_end[1]);
-      cur_N = job == 0 ? p.g_N[0] : (job == 1 ? p.g_N[1] : p.g_N[2]);
-      const int tn = (cur_N + BN - 1) / BN, tl = tile - t0, tmg = tl / tn;
-      n0 = (tl - tmg * tn) * BN;
-      row0 = tmg * kBM;
-      rows = min(kBM, p.M - row0);
-      slot = -1;
-      return;
-    }
     int tm = tile / tiles_n;
     n0 = (tile - tm * tiles_n) * BN;
     if (EPI == EPI_SHRINK && n_jobs > 1) {
@@ -207,7 +179,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (kb < nkb_main) {
             const CUtensorMap* ma = &tmA;
             const CUtensorMap* mb = &tmB;
-            if ((EPI == EPI_SHRINK || EPI == EPI_STORE_GROUP) && job > 0) {
+            if (EPI == EPI_SHRINK && job > 0) {
               ma = (job == 1) ? &tmA2 : &tmA3;
               mb = (job == 1) ? &tmB2 : &tmB3;
             }
@@ -276,7 +248,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int ncols = (EPI == EPI_SHRINK) ? min(BN, (p.N + 31) / 32 * 32) : BN;
 #pragma unroll 1
       for (int c = 0; c < ncols; c += 32) {
-        if (n0 + c >= cur_N) break;
+        if (n0 + c >= p.N) break;
         uint32_t v[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c, v);
         tmem_ld_wait();
@@ -300,25 +272,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               }
             }
           }
-        } else if (row_ok && (EPI == EPI_STORE || EPI == EPI_STORE_GROUP || slot >= 0)) {
+        } else if (row_ok && (EPI == EPI_STORE || slot >= 0)) {
           const float sc = (EPI == EPI_SHRINK) ? p.scale : 1.f;
           __nv_bfloat16* ybase = p.y;
           __nv_bfloat16* ylo_base = p.y_lo;
-          float* y0base = p.y0;
-          int ldy = p.ldy;
-          if (EPI == EPI_STORE_GROUP) {
-            ybase = (job == 0) ? p.g_y[0] : (job == 1) ? p.g_y[1] : p.g_y[2];
-            y0base = (job == 0) ? p.g_y0[0] : (job == 1) ? p.g_y0[1] : p.g_y0[2];
-            ldy = cur_N;
-          }
           if (EPI == EPI_SHRINK && p.n_jobs > 0) {
             ybase = (job == 0) ? p.ys[0] : (job == 1) ? p.ys[1] : p.ys[2];
             ylo_base = (job == 0) ? p.ys_lo[0] : (job == 1) ? p.ys_lo[1] : p.ys_lo[2];
           }
-          __nv_bfloat16* yrow = ybase + grow * (size_t)ldy + n0 + c;
+          __nv_bfloat16* yrow = ybase + grow * (size_t)p.ldy + n0 + c;
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
-            if (n0 + c + j < cur_N) {  // N is a multiple of 8
+            if (n0 + c + j < p.N) {  // N is a multiple of 8
               float f[8];
 #pragma unroll
               for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]) * sc;
@@ -334,10 +299,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 l.y = pack_bf16(f[2] - bf16_lo(o.y), f[3] - bf16_hi(o.y));
                 l.z = pack_bf16(f[4] - bf16_lo(o.z), f[5] - bf16_hi(o.z));
                 l.w = pack_bf16(f[6] - bf16_lo(o.w), f[7] - bf16_hi(o.w));
-                *reinterpret_cast<uint4*>(ylo_base + grow * (size_t)ldy + n0 + c + j) = l;
+                *reinterpret_cast<uint4*>(ylo_base + grow * (size_t)p.ldy + n0 + c + j) = l;
               }
-              if ((EPI == EPI_STORE || EPI == EPI_STORE_GROUP) && y0base) {
-                float* y0row = y0base + grow * (size_t)ldy + n0 + c + j;
+              if (EPI == EPI_STORE && p.y0) {
+                float* y0row = p.y0 + grow * (size_t)p.ldy + n0 + c + j;
                 *reinterpret_cast<uint4*>(y0row) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                 *reinterpret_cast<uint4*>(y0row + 4) = make_uint4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
               }
@@ -425,25 +390,11 @@ static moin_status launch_cfg(HostState* hs, const CUtensorMap& a, const CUtenso
                               const CUtensorMap& a3, const CUtensorMap& b2, const TcParams& p, long max_tiles,
                               cudaStream_t stream, const CUtensorMap* b3 = nullptr) {
   using Cfg = TcCfg<BN>;
-  constexpr int bn_idx = (BN == 256 ? 2 : BN == 128 ? 1 : 0);
-  constexpr int slot = (EPI == EPI_STORE_GROUP) ? OPTIN_TC_GROUP + bn_idx : OPTIN_TC_GEMM + 4 * bn_idx + EPI;
+  constexpr int slot = OPTIN_TC_GEMM + 4 * (BN == 256 ? 2 : BN == 128 ? 1 : 0) + EPI;
   cudaError_t e = ensure_smem_optin(slot, tc_gemm_kernel<BN, EPI>, Cfg::kSmemBytes);
   if (e != cudaSuccess) return record_cuda(e);
   long grid = max_tiles < hs->n_sms ? max_tiles : hs->n_sms;
   if (grid < 1) grid = 1;
-  if (EPI == EPI_STORE_GROUP) {   // may start while the kernel before it on the stream drains (it waits for it itself)
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(kTcThreads);
-    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return record_cuda(cudaLaunchKernelEx(&cfg, tc_gemm_kernel<BN, EPI>, a, b, a2, a3, b2, b3 ? *b3 : b2, p));
-  }
   tc_gemm_kernel<BN, EPI><<<(int)grid, kTcThreads, Cfg::kSmemBytes, stream>>>(a, b, a2, a3, b2, b3 ? *b3 : b2, p);
   return record_cuda(cudaGetLastError());
 }
@@ -481,9 +432,13 @@ bool tc_router_supported(int Q, int K, int D) { return Q >= 1 && K >= 1 && D >= 
 bool tc_fused_supported(int r) { return r >= 8 && r <= 128 && (r % 8) == 0; }
 
 moin_status launch_tc_gemm(HostState* hs, const __nv_bfloat16* x, const __nv_bfloat16* W, __nv_bfloat16* y, float* y0,
-                           int T, int d_in, int d_out, cudaStream_t stream) {
+                           int T, int d_in, int d_out, cudaStream_t stream, int cta_budget) {
   const long tiles_m = (T + kBM - 1) / kBM;
-  const int bn = (tiles_m <= 2 && y0 != nullptr) ? pick_bn_small_m(d_out, d_in) : pick_bn(tiles_m, d_out, hs->n_sms);
+  int bn = (tiles_m <= 2 && y0 != nullptr) ? pick_bn_small_m(d_out, d_in) : pick_bn(tiles_m, d_out, hs->n_sms);
+  // Beside the adapter streams (decode): a CTA of this kernel keeps its SM to itself (the ring takes the shared
+  // memory), and while a launch still has CTAs waiting for an SM the stream kernel behind it gets none.  Widen the
+  // tiles until the launch fits the share of the SMs the caller grants it.
+  while (cta_budget > 0 && bn < 256 && d_out >= 2 * bn && tiles_m * ((d_out + bn - 1) / bn) > cta_budget) bn *= 2;
   CUtensorMap a, b;
   moin_status st = make_map(&a, x, T, d_in, kBM);
   if (!st) st = make_map(&b, W, d_out, d_in, bn);
@@ -494,42 +449,6 @@ moin_status launch_tc_gemm(HostState* hs, const __nv_bfloat16* x, const __nv_bfl
   if (bn == 256) return launch_cfg<256, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream);
   if (bn == 128) return launch_cfg<128, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream);
   return launch_cfg<64, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream);
-}
-
-// Base GEMMs of up to kMaxStoreJobs projections that share T and d_in (decode-sized batches): one launch.
-moin_status launch_tc_gemm_group(HostState* hs, const __nv_bfloat16* const* xs, const __nv_bfloat16* const* Ws,
-                                 __nv_bfloat16* const* ys, float* const* y0s, const int* d_outs, int n_jobs, int T,
-                                 int d_in, cudaStream_t stream) {
-  if (n_jobs < 1 || n_jobs > kMaxStoreJobs) return MOIN_ERR_INVALID_ARG;
-  const long tiles_m = (T + kBM - 1) / kBM;
-  int widest = 0;
-  for (int j = 0; j < n_jobs; ++j) widest = d_outs[j] > widest ? d_outs[j] : widest;
-  const int bn = tiles_m <= 2 ? pick_bn_small_m(widest, d_in) : pick_bn(tiles_m, widest, hs->n_sms);
-  CUtensorMap a[kMaxStoreJobs], b[kMaxStoreJobs];
-  TcParams p = {};
-  p.M = T; p.K = d_in; p.N = widest; p.scale = 1.f; p.status = hs->status; p.g_n = n_jobs;
-  int tiles = 0;
-  for (int j = 0; j < n_jobs; ++j) {
-    moin_status st = make_map(&a[j], xs[j], T, d_in, kBM);
-    if (!st) st = make_map(&b[j], Ws[j], d_outs[j], d_in, bn);
-    if (st) return st;
-    tiles += (int)tiles_m * ((d_outs[j] + bn - 1) / bn);
-    p.g_N[j] = d_outs[j];
-    p.g_tile_end[j] = tiles;
-    p.g_y[j] = ys[j];
-    p.g_y0[j] = y0s[j];
-  }
-  for (int j = n_jobs; j < kMaxStoreJobs; ++j) {
-    a[j] = a[0];
-    b[j] = b[0];
-    p.g_N[j] = p.g_N[0];
-    p.g_tile_end[j] = tiles;
-    p.g_y[j] = p.g_y[0];
-    p.g_y0[j] = p.g_y0[0];
-  }
-  if (bn == 256) return launch_cfg<256, EPI_STORE_GROUP>(hs, a[0], b[0], a[1], a[2], b[1], p, tiles, stream, &b[2]);
-  if (bn == 128) return launch_cfg<128, EPI_STORE_GROUP>(hs, a[0], b[0], a[1], a[2], b[1], p, tiles, stream, &b[2]);
-  return launch_cfg<64, EPI_STORE_GROUP>(hs, a[0], b[0], a[1], a[2], b[1], p, tiles, stream, &b[2]);
 }
 
 moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,

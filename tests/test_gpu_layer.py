@@ -37,17 +37,9 @@ def test_tiny_config_routed_by_the_router():
     assert_layer_close(y, oracle_layer(case), "tiny routed")
 
 
-@pytest.fixture(params=[1, 2, 3], ids=["two-launch", "tma", "fused"])
-def stream_impl(request):
-    """Every implementation of the short-segment kernels (separate shrink / expand launches, TMA-staged, fused launch)."""
-    moin.set_option(moin.OPT_STREAM_IMPL, request.param)
-    yield request.param
-    moin.set_option(moin.OPT_STREAM_IMPL, 0)
-
-
 @pytest.mark.parametrize("r", [8, 16, 24, 32, 40, 48, 56, 64, 72, 96, 120, 128])
 @pytest.mark.parametrize("mode", MODES)
-def test_every_supported_rank(r, mode, stream_impl):
+def test_every_supported_rank(r, mode):
     rng = mi.np_rng(7, r)
     # ragged T, d_out not a multiple of 16 or 64; d_in alternates between a multiple of 256 and not
     E, T, d_in, d_out = 6, 333, (192 if r % 16 else 512), 328
@@ -60,7 +52,7 @@ def test_every_supported_rank(r, mode, stream_impl):
 
 
 @pytest.mark.parametrize("mode", MODES)
-def test_base_only_and_missing_adapters(mode, stream_impl):
+def test_base_only_and_missing_adapters(mode):
     pool = mi.make_pool(5, 16, 256, 128, 8, 1, missing=(1, 3))
     te = np.array([-1, 1, 3, 0, 2, 4, 99, -5] * 20, np.int32)
     case = mi.layer_case("fallback", len(te), 256, 128, pool, te, 2.0, 8, 2)
@@ -97,7 +89,7 @@ def test_long_runs_at_rank_128_through_the_fused_gemm():
     assert_layer_close(y, oracle_layer(case), "rank 128 long runs")
 
 
-def test_decode_config_all_projections(stream_impl):
+def test_decode_config_all_projections():
     # 256 single-token requests, 500 rank-64 experts: every token checked against the oracle.
     cases = mi.decode_batch(seed=1, device=DEV)
     te = cases[0].token_expert
@@ -124,7 +116,7 @@ def test_prefill_config_sampled_rows():
 
 
 @pytest.mark.parametrize("mode", MODES)
-def test_request_permutation_and_determinism(mode, stream_impl):
+def test_request_permutation_and_determinism(mode):
     # experts do not interact: permuting requests permutes output rows (bitwise), and reruns are bitwise equal
     pool = mi.make_pool(12, 32, 256, 256, 9, 1)
     rng = mi.np_rng(9, 2)
@@ -145,7 +137,7 @@ def test_request_permutation_and_determinism(mode, stream_impl):
 
 
 @pytest.mark.parametrize("mode", MODES)
-def test_grouped_projections_equal_single_calls(mode, stream_impl):
+def test_grouped_projections_equal_single_calls(mode):
     # {q,k,v}-like group: shared plan, different shapes; the group's outputs are bit-identical to one call per
     # projection, and match the oracle.
     rng = mi.np_rng(13, 1)

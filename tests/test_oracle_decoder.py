@@ -152,7 +152,8 @@ def np_round_bf16(a: np.ndarray) -> np.ndarray:
     return r.view(np.float64).reshape(a.shape)
 
 
-def np_block_storage_rounded(model: mi.DecoderModel, layer: int, x: np.ndarray, expert: int) -> np.ndarray:
+def np_block_storage_rounded(model: mi.DecoderModel, layer: int, x: np.ndarray, expert) -> np.ndarray:
+    """`expert`: one id for the whole request, or one id per token (array of the request's length)."""
     c = model.cfg
     rb = np_round_bf16
     f64 = lambda t: t.to(torch.float64).numpy()
@@ -160,12 +161,16 @@ def np_block_storage_rounded(model: mi.DecoderModel, layer: int, x: np.ndarray, 
     def norm(v, gain):
         return rb(v / np.sqrt((v * v).mean(axis=1, keepdims=True) + c.rms_eps) * f64(gain)[None, :])
 
+    experts = np.full(x.shape[0], expert, np.int64) if np.ndim(expert) == 0 else np.asarray(expert, np.int64)
+
     def proj(name, v):
         y = v @ f64(model.W[layer][name]).T
         pool = model.pools[layer][name]
-        s = int(pool.slot_of_expert[expert]) if expert >= 0 else -1
-        if s >= 0:
-            y = y + c.scale * ((v @ f64(pool.A[s]).T) @ f64(pool.B[s]).T)   # h stays unrounded
+        for e in np.unique(experts):
+            s = int(pool.slot_of_expert[e]) if e >= 0 else -1
+            if s >= 0:
+                rows = experts == e
+                y[rows] = y[rows] + c.scale * ((v[rows] @ f64(pool.A[s]).T) @ f64(pool.B[s]).T)   # h stays unrounded
         return rb(y)
 
     def rope(v, n_h):
@@ -222,3 +227,47 @@ def test_storage_rounded_variant_rounds_exactly_at_the_listed_points(setup):
     f64 = lambda t: t.to(torch.float64).numpy()
     xn = np_round_bf16(hidden / np.sqrt((hidden * hidden).mean(axis=1, keepdims=True) + c.rms_eps) * f64(model.final_norm)[None, :])
     np.testing.assert_allclose(got, np_round_bf16(xn @ f64(model.lm_head).T), rtol=1e-9, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------
+# One expert per token (the paper's future-work variant, Sec. 5 "per-token adapters"; Sec. 3.3 uses one per
+# request).  Pins: ids that are constant inside every request give the per-request result bit for bit; with mixed
+# ids, every token's projections follow its own adapter (numpy restatement of a block, exact and storage-rounded);
+# a token without adapter inside a routed request gets the base projections.
+# ---------------------------------------------------------------------------------------------
+def test_per_token_experts_constant_per_request_equal_per_request_experts(setup):
+    model, batch, orc = setup
+    cu = batch.cu_seqlens.numpy()
+    re_ = batch.req_expert.numpy()
+    te = np.repeat(re_, np.diff(cu)).astype(np.int32)
+    for rs in (False, True):
+        a = orc.forward(batch.tokens.numpy(), cu, re_, round_storage=rs, want_hidden=True)
+        b = orc.forward(batch.tokens.numpy(), cu, None, round_storage=rs, want_hidden=True, token_expert=te)
+        assert np.array_equal(a["logits"], b["logits"]) and np.array_equal(a["hidden"], b["hidden"])
+
+
+def test_per_token_experts_follow_each_tokens_adapter(setup):
+    model, batch, orc = setup
+    c = model.cfg
+    cu = batch.cu_seqlens.numpy()
+    rng = np.random.default_rng(5)
+    te = rng.integers(-1, c.E, size=batch.T).astype(np.int32)        # -1 and the adapter-less expert 2 included
+    hidden = mi.bf16_to_f64(model.embed)[batch.tokens.numpy()]
+    args = (batch.tokens.numpy(), cu, None)
+    for layer in range(c.n_layers):
+        got = orc.forward(*args, layer_begin=layer, layer_end=layer + 1, hidden_in=hidden, round_storage=True,
+                          want_hidden=True, want_logits=False, token_expert=te)["hidden"]
+        ref = np.concatenate([np_block_storage_rounded(model, layer, hidden[cu[r]:cu[r + 1]], te[cu[r]:cu[r + 1]])
+                              for r in range(batch.R)])
+        np.testing.assert_allclose(got, ref, rtol=1e-9, atol=1e-12)
+        hidden = got
+    # the ids matter: the same tokens with every id set to its request's first id give something else
+    te_first = np.repeat(te[cu[:-1]], np.diff(cu)).astype(np.int32)
+    a = orc.forward(*args, token_expert=te)["logits"]
+    b = orc.forward(*args, token_expert=te_first)["logits"]
+    assert np.abs(a - b).max() > 1e-3
+    # and a token's result does not depend on ids of LATER tokens of its request (causal attention, per-row adapters)
+    te2 = te.copy()
+    te2[cu[2] + 9:cu[3]] = 0
+    b2 = orc.forward(*args, token_expert=te2)["logits"]
+    assert np.array_equal(a[cu[2]:cu[2] + 9], b2[cu[2]:cu[2] + 9])

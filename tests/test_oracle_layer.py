@@ -151,3 +151,68 @@ def test_golden_adapter_parameter_share():
     assert total == int(vals["adapter_parameters"])
     share = total / vals["base_parameters"]
     assert abs(share - vals["paper_share"]) < 0.015
+
+
+# ---------------------------------------------------------------------------------------------
+# Variants from the paper's future-work list (Sec. 5): a rank per topic ("adaptive rank") and a function
+# between the two low-rank matrices.  Same kind of pins as above.
+# ---------------------------------------------------------------------------------------------
+def test_per_slot_rank_equals_merged_weight_of_the_truncated_adapter():
+    x, W, A, B, te, slot = _case(T=64, r=16)
+    ranks = np.array([16, 8, 0, 12, 5], np.int32)          # slot -> rank (0: the adapter contributes nothing)
+    y = oracle.lora_linear(x, W, A, B, te, slot, 2.0, slot_rank=ranks)
+    for e in np.unique(te):
+        rows = np.nonzero(te == e)[0]
+        k = ranks[slot[e]]
+        merged = W + 2.0 * (B[slot[e]][:, :k] @ A[slot[e]][:k, :])
+        np.testing.assert_allclose(y[rows], x[rows] @ merged.T, rtol=0, atol=1e-12)
+    # full rank for every slot = no rank table at all, bit for bit
+    assert np.array_equal(oracle.lora_linear(x, W, A, B, te, slot, 2.0, slot_rank=np.full(5, 16, np.int32)),
+                          oracle.lora_linear(x, W, A, B, te, slot, 2.0))
+    # what is stored beyond a slot's rank is never read: poison it
+    A2, B2 = A.copy(), B.copy()
+    for s_, k in enumerate(ranks):
+        A2[s_, k:, :] = np.nan
+        B2[s_, :, k:] = np.inf
+    assert np.array_equal(oracle.lora_linear(x, W, A2, B2, te, slot, 2.0, slot_rank=ranks), y)
+
+
+@pytest.mark.parametrize("act,fn", [(oracle.ACT_RELU, lambda h: np.maximum(h, 0.0)),
+                                    (oracle.ACT_SILU, lambda h: h / (1.0 + np.exp(-h))),
+                                    (oracle.ACT_GELU, None)])
+def test_activation_between_the_low_rank_matrices(act, fn):
+    import math
+    if fn is None:
+        fn = np.vectorize(lambda v: 0.5 * v * (1.0 + math.erf(v / math.sqrt(2.0))))
+    x, W, A, B, te, slot = _case(T=50, missing=(3,))
+    y = oracle.lora_linear(x, W, A, B, te, slot, 1.5, act=act)
+    for t in range(x.shape[0]):
+        ref = W @ x[t]
+        if slot[te[t]] >= 0:
+            ref = ref + 1.5 * (B[slot[te[t]]] @ fn(A[slot[te[t]]] @ x[t]))
+        np.testing.assert_allclose(y[t], ref, rtol=0, atol=1e-12)
+    # no activation = the paper's layer, bit for bit; and the activation does change routed rows only
+    y0 = oracle.lora_linear(x, W, A, B, te, slot, 1.5)
+    assert np.array_equal(oracle.lora_linear(x, W, A, B, te, slot, 1.5, act=oracle.ACT_NONE), y0)
+    routed = slot[te] >= 0
+    assert np.abs(y - y0)[routed].max() > 1e-3 and np.array_equal(y[~routed], y0[~routed])
+
+
+def test_relu_rank_one_closed_form_and_rank_with_activation():
+    # r = 1 with ReLU: the low-rank term is s * max(a . x, 0) * b - it vanishes exactly where a . x < 0
+    x, W, A, B, te, slot = _case(r=1)
+    y = oracle.lora_linear(x, W, A, B, te, slot, 0.5, act=oracle.ACT_RELU)
+    base = oracle.lora_linear(x, W, None, None, None, None, 0.5)
+    for t in range(x.shape[0]):
+        a, b = A[slot[te[t]], 0], B[slot[te[t]], :, 0]
+        np.testing.assert_allclose(y[t], base[t] + 0.5 * max(a @ x[t], 0.0) * b, rtol=0, atol=1e-12)
+        if a @ x[t] < 0:
+            assert np.array_equal(y[t], base[t])
+    # rank table and activation together: SiLU is applied to the rows the slot has, the others are not read
+    x, W, A, B, te, slot = _case(T=40, r=8)
+    ranks = np.array([8, 3, 8, 1, 6], np.int32)
+    y = oracle.lora_linear(x, W, A, B, te, slot, 2.0, slot_rank=ranks, act=oracle.ACT_SILU)
+    for t in range(x.shape[0]):
+        s_, k = slot[te[t]], ranks[slot[te[t]]]
+        h = A[s_][:k] @ x[t]
+        np.testing.assert_allclose(y[t], W @ x[t] + 2.0 * (B[s_][:, :k] @ (h / (1.0 + np.exp(-h)))), rtol=0, atol=1e-12)
