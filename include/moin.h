@@ -183,7 +183,18 @@ moin_status moin_route_static(const moin_router* router, const void* queries, in
  *   A[n_slots, r, d_in] = W_a,  B[n_slots, d_out, r] = W_b,
  * and slot_of_expert[E] maps an expert id to its slot, -1 = the expert has no adapter
  * (paper Sec. 4: then the base model alone is used).
+ *
+ * Two optional members cover variants from the paper's future-work list (Sec. 5); zero / NULL gives the paper's
+ * layer.  A caller that fills the struct member by member should zero it first.
+ *   slot_rank   "adaptive rank": a rank per topic.  slot_rank[s] (device, [n_slots] int32, a multiple of 8 in
+ *               [0, r]) is the rank of slot s; r stays the STORED rank (row count of A[s], row pitch of B[s]).
+ *               Only the first slot_rank[s] rows of A[s] and columns of B[s] enter the result, and the kernels
+ *               that stream adapters read nothing beyond them, so a low-rank topic costs proportionally fewer
+ *               bytes.  What is stored beyond a slot's rank must be finite (the tensor-core path may multiply
+ *               it by zero).  NULL: every slot has rank r.
+ *   activation  a function applied between the two matrices: y = W x + s W_b act(W_a x); MOIN_ACT_*.
  * ------------------------------------------------------------------------------------- */
+enum { MOIN_ACT_NONE = 0, MOIN_ACT_RELU = 1, MOIN_ACT_SILU = 2, MOIN_ACT_GELU = 3 /* 0.5 v (1 + erf(v / sqrt 2)) */ };
 typedef struct {
   const void* A;
   const void* B;
@@ -193,6 +204,8 @@ typedef struct {
   int32_t r;     /* LoRA rank: multiple of 8, 8..128 (128 is the rank of the paper's experts, Sec. 4) */
   int32_t d_in;  /* multiple of 64 */
   int32_t d_out; /* multiple of 8 */
+  int32_t activation;            /* MOIN_ACT_*; 0 = none (the paper's formula) */
+  const int32_t* slot_rank;      /* device [n_slots] or NULL */
 } moin_pool;
 
 /* ---------------------------------------------------------------------------------------

@@ -6,9 +6,9 @@ library is missing or no sm_100 GPU is present, calls raise.
 """
 from .binding import (MoinError, Router, Pool, Plan, DecoderModel, lib, lib_path, route, route_top2, route_static, ROUTE_STATIC_MAX_Q, plan_build, kmeans_update, AdapterCache, lora_linear, lora_linear_group, JobGroup,
                       decoder_forward, device_status, device_status_reset, selftest_bounded_wait, set_option, profile_enable, profile_read, PLAN_AUTO, PLAN_SEGMENTS,
-                      PLAN_TILES, LOGITS_ALL, LOGITS_LAST, LOGITS_NONE, OPT_GEMM_IMPL, EXPORTED_SYMBOLS)
+                      PLAN_TILES, LOGITS_ALL, LOGITS_LAST, LOGITS_NONE, OPT_GEMM_IMPL, ACT_NONE, ACT_RELU, ACT_SILU, ACT_GELU, EXPORTED_SYMBOLS)
 
 __all__ = ["MoinError", "Router", "Pool", "Plan", "DecoderModel", "lib", "lib_path", "route", "route_top2", "route_static", "ROUTE_STATIC_MAX_Q", "plan_build", "kmeans_update", "AdapterCache",
            "lora_linear", "lora_linear_group", "JobGroup", "decoder_forward", "device_status", "device_status_reset", "selftest_bounded_wait", "set_option", "profile_enable", "profile_read", "PLAN_AUTO",
-           "PLAN_SEGMENTS", "PLAN_TILES", "LOGITS_ALL", "LOGITS_LAST", "LOGITS_NONE", "OPT_GEMM_IMPL",
+           "PLAN_SEGMENTS", "PLAN_TILES", "LOGITS_ALL", "LOGITS_LAST", "LOGITS_NONE", "OPT_GEMM_IMPL", "ACT_NONE", "ACT_RELU", "ACT_SILU", "ACT_GELU",
            "EXPORTED_SYMBOLS"]

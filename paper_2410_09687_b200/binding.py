@@ -15,6 +15,7 @@ _lib: Optional[ctypes.CDLL] = None
 PLAN_AUTO, PLAN_SEGMENTS, PLAN_TILES = 0, 1, 2
 LOGITS_ALL, LOGITS_LAST, LOGITS_NONE = 0, 1, 2
 OPT_GEMM_IMPL = 1
+ACT_NONE, ACT_RELU, ACT_SILU, ACT_GELU = 0, 1, 2, 3
 
 EXPORTED_SYMBOLS = (
     "moin_status_string", "moin_version", "moin_last_cuda_error", "moin_device_status", "moin_device_status_reset",
@@ -39,7 +40,7 @@ class _Router(ctypes.Structure):
 class _Pool(ctypes.Structure):
     _fields_ = [("A", ctypes.c_void_p), ("B", ctypes.c_void_p), ("slot_of_expert", ctypes.c_void_p),
                 ("E", ctypes.c_int32), ("n_slots", ctypes.c_int32), ("r", ctypes.c_int32), ("d_in", ctypes.c_int32),
-                ("d_out", ctypes.c_int32)]
+                ("d_out", ctypes.c_int32), ("activation", ctypes.c_int32), ("slot_rank", ctypes.c_void_p)]
 
 
 class _Job(ctypes.Structure):
@@ -336,14 +337,17 @@ def kmeans_update(plan: "Plan", x: torch.Tensor, centroids_old: torch.Tensor,
 class Pool:
     """moin_pool: stacked adapters of one projection."""
 
-    def __init__(self, A: torch.Tensor, B: torch.Tensor, slot_of_expert: torch.Tensor):
+    def __init__(self, A: torch.Tensor, B: torch.Tensor, slot_of_expert: torch.Tensor,
+                 slot_rank: Optional[torch.Tensor] = None, activation: int = ACT_NONE):
         assert A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16 and slot_of_expert.dtype == torch.int32
-        self.A, self.B, self.slot_of_expert = A, B, slot_of_expert
+        assert slot_rank is None or (slot_rank.dtype == torch.int32 and slot_rank.shape[0] == A.shape[0])
+        self.A, self.B, self.slot_of_expert, self.slot_rank, self.activation = A, B, slot_of_expert, slot_rank, activation
         n_slots, r, d_in = A.shape
         d_out = B.shape[1]
         assert B.shape[0] == n_slots and B.shape[2] == r
         self.E, self.n_slots, self.r, self.d_in, self.d_out = slot_of_expert.shape[0], n_slots, r, d_in, d_out
-        self.c = _Pool(_ptr(A), _ptr(B), _ptr(slot_of_expert), self.E, n_slots, r, d_in, d_out)
+        self.c = _Pool(_ptr(A), _ptr(B), _ptr(slot_of_expert), self.E, n_slots, r, d_in, d_out, int(activation),
+                       _ptr(slot_rank))
 
 
 class Plan:

@@ -466,6 +466,7 @@ static moin_status check_job(const moin_plan* plan, const void* x, const void* W
     if (*r < 8 || *r > 128 || (*r % 8) != 0) return MOIN_ERR_UNSUPPORTED_RANK;
     if (!pool->A || !pool->B || !pool->slot_of_expert || !plan->buffer) return MOIN_ERR_INVALID_ARG;
     if (pool->E != plan->E) return MOIN_ERR_INVALID_ARG;
+    if (pool->activation < MOIN_ACT_NONE || pool->activation > MOIN_ACT_GELU) return MOIN_ERR_INVALID_ARG;
     if (!aligned16(pool->A) || !aligned16(pool->B)) return MOIN_ERR_MISALIGNED;
     if (plan->mode != MOIN_PLAN_SEGMENTS && plan->mode != MOIN_PLAN_TILES) return MOIN_ERR_INVALID_ARG;
   }
@@ -529,7 +530,8 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
         const __nv_bfloat16* gx[kTcMaxShrinkJobs];
         __nv_bfloat16* gh[kTcMaxShrinkJobs];
         int n = 0;
-        while (j0 + n < n_jobs && n < kTcMaxShrinkJobs && d_in[j0 + n] == d_in[j0] && r[j0 + n] == r[j0]) {
+        while (j0 + n < n_jobs && n < kTcMaxShrinkJobs && d_in[j0 + n] == d_in[j0] && r[j0 + n] == r[j0] &&
+               jobs[j0 + n].pool->activation == jobs[j0].pool->activation) {
           gp[n] = jobs[j0 + n].pool;
           gx[n] = (const __nv_bfloat16*)jobs[j0 + n].x;
           gh[n] = reinterpret_cast<__nv_bfloat16*>(ws_job[j0 + n]);
@@ -582,6 +584,7 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
       sj.A[j] = (const __nv_bfloat16*)jobs[j].pool->A;
       sj.h[j] = h[j];
       sj.slot_of_expert[j] = jobs[j].pool->slot_of_expert;
+      sj.slot_rank[j] = jobs[j].pool->slot_rank;
       sj.r[j] = r[j];
       sj.d_in[j] = d_in[j];
     }
@@ -604,6 +607,8 @@ moin_status moin_lora_linear_group(const moin_plan* plan, const moin_lora_job* j
     ej.y0[j] = y0[j];
     ej.y[j] = (__nv_bfloat16*)jobs[j].y;
     ej.slot_of_expert[j] = jobs[j].pool->slot_of_expert;
+    ej.slot_rank[j] = jobs[j].pool->slot_rank;
+    ej.act[j] = jobs[j].pool->activation;
     ej.r[j] = r[j];
     ej.d_out[j] = d_out[j];
   }

@@ -101,6 +101,16 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// Function between the two low-rank matrices (MOIN_ACT_*).
+__device__ __forceinline__ float lora_act(float v, int act) {
+  switch (act) {
+    case MOIN_ACT_RELU: return fmaxf(v, 0.f);
+    case MOIN_ACT_SILU: return v / (1.f + __expf(-v));
+    case MOIN_ACT_GELU: return 0.5f * v * (1.f + erff(v * 0.70710678118654752f));
+    default: return v;
+  }
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -118,6 +128,7 @@ struct ShrinkJobs {
   const __nv_bfloat16* A[kMaxStreamJobs];
   float* h[kMaxStreamJobs];
   const int* slot_of_expert[kMaxStreamJobs];
+  const int* slot_rank[kMaxStreamJobs];   // per-slot rank (nullptr: the pool's r)
   int r[kMaxStreamJobs], d_in[kMaxStreamJobs], per_seg[kMaxStreamJobs];
   int n;
 };
@@ -127,6 +138,8 @@ struct ExpandJobs {
   const float* y0[kMaxStreamJobs];
   __nv_bfloat16* y[kMaxStreamJobs];
   const int* slot_of_expert[kMaxStreamJobs];
+  const int* slot_rank[kMaxStreamJobs];   // per-slot rank (nullptr: the pool's r)
+  int act[kMaxStreamJobs];                // MOIN_ACT_* applied to h
   int r[kMaxStreamJobs], d_out[kMaxStreamJobs], rows_per_item[kMaxStreamJobs], per_seg[kMaxStreamJobs];
   int n;
 };

@@ -50,15 +50,17 @@ __device__ __forceinline__ ItemRef decode_item(int item, int nseg, const Jobs& j
   return it;
 }
 
-struct SegMeta { int slot, s0, n, job, sub; };
+struct SegMeta { int slot, s0, n, job, sub, r_use; };   // r_use: rank of the slot's adapter (<= the stored rank)
 template <class Jobs>
 __device__ __forceinline__ SegMeta load_seg(const int4* __restrict__ seg_tab, const Jobs& jobs, int item, int items,
                                             int nseg) {
-  SegMeta m = {-1, 0, 0, 0, 0};
+  SegMeta m = {-1, 0, 0, 0, 0, 0};
   if (item < items) {
     const ItemRef it = decode_item(item, nseg, jobs);
     const int4 e = __ldg(seg_tab + it.seg);   // (expert, start, length, -)
     m.slot = __ldg(pick(jobs.slot_of_expert, it.job) + e.x);
+    const int* rank_tab = pick(jobs.slot_rank, it.job);
+    m.r_use = (m.slot >= 0 && rank_tab) ? min(__ldg(rank_tab + m.slot), pick(jobs.r, it.job)) : pick(jobs.r, it.job);
     m.s0 = e.y;
     m.n = e.z;
     m.job = it.job;
@@ -89,14 +91,14 @@ lora_shrink_stream_kernel(const int* __restrict__ header, const int* __restrict_
   for (; item < items; item += gridDim.x) {
     const SegMeta cur = nxt;
     nxt = load_seg(seg_tab, jobs, item + gridDim.x, items, nseg);  // lookahead
-    if (cur.slot < 0) continue;  // uniform per CTA
+    if (cur.slot < 0 || cur.sub * 16 >= cur.r_use) continue;  // uniform per CTA: no adapter, or rows beyond its rank
     const int r = pick(jobs.r, cur.job), d_in = pick(jobs.d_in, cur.job);
     const __nv_bfloat16* __restrict__ x = pick(jobs.x, cur.job);
     const __nv_bfloat16* __restrict__ A = pick(jobs.A, cur.job);
     float* __restrict__ h = pick(jobs.h, cur.job);
     const int steps = d_in >> 5;  // 32 k per step
     const int rho0 = cur.sub * 16 + g, rho1 = rho0 + 8;
-    const bool v0 = rho0 < r, v1 = rho1 < r;
+    const bool v0 = rho0 < cur.r_use, v1 = rho1 < cur.r_use;   // rows beyond the slot's rank are not read
     const __nv_bfloat16* a_row0 = A + ((size_t)cur.slot * r + (v0 ? rho0 : 0)) * (size_t)d_in + 8 * t;
     const __nv_bfloat16* a_row1 = A + ((size_t)cur.slot * r + (v1 ? rho1 : 0)) * (size_t)d_in + 8 * t;
     for (int tc = 0; tc < cur.n; tc += 8) {
@@ -186,6 +188,11 @@ lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict_
     int slots[kMaxStreamJobs];
 #pragma unroll
     for (int j = 0; j < kMaxStreamJobs; ++j) slots[j] = (j < jobs.n) ? __ldg(jobs.slot_of_expert[j] + e.x) : -1;
+    int ranks[kMaxStreamJobs];   // rank of the slot's adapter: columns of B and entries of h beyond it are not read
+#pragma unroll
+    for (int j = 0; j < kMaxStreamJobs; ++j)
+      ranks[j] = (j < jobs.n && slots[j] >= 0 && jobs.slot_rank[j]) ? min(__ldg(jobs.slot_rank[j] + slots[j]), jobs.r[j])
+                                                                     : (j < jobs.n ? jobs.r[j] : 0);
     const int row_first = (g < n) ? __ldg(perm + s0 + g) : -1;
     const long long seg_end = (long long)(seg + 1) * tps;
     int rem = (int)(u - (long long)seg * tps);
@@ -206,6 +213,7 @@ lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict_
       const int slot = pick(slots, job);
       if (slot >= 0) {
         const int r = pick(jobs.r, job), d_out = pick(jobs.d_out, job);
+        const int r_use = pick(ranks, job), act = pick(jobs.act, job);
         const float* __restrict__ h = pick(jobs.h, job);
         const float* __restrict__ y0 = pick(jobs.y0, job);
         __nv_bfloat16* __restrict__ y = pick(jobs.y, job);
@@ -219,7 +227,7 @@ lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict_
           for (int p = 0; p < P; ++p) {
             const int rb = 32 * p + 8 * t;
             float v[8];
-            if (vx && rb < r) {
+            if (vx && rb < r_use) {
               const float4 f0 = *reinterpret_cast<const float4*>(h + (size_t)(s0 + tc + g) * r + rb);
               const float4 f1 = *reinterpret_cast<const float4*>(h + (size_t)(s0 + tc + g) * r + rb + 4);
               v[0] = f0.x; v[1] = f0.y; v[2] = f0.z; v[3] = f0.w; v[4] = f1.x; v[5] = f1.y; v[6] = f1.z; v[7] = f1.w;
@@ -229,7 +237,7 @@ lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict_
             }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              const float s0v = v[2 * q] * scale, s1v = v[2 * q + 1] * scale;
+              const float s0v = lora_act(v[2 * q], act) * scale, s1v = lora_act(v[2 * q + 1], act) * scale;
               const uint32_t hi = pack_bf16(s0v, s1v);
               hh[p][q] = hi;
               hl[p][q] = pack_bf16(s0v - bf16_lo(hi), s1v - bf16_hi(hi));
@@ -248,8 +256,8 @@ lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict_
               for (int p = 0; p < P; ++p) {
                 const int rb = 32 * p + 8 * t;
                 const uint4 z = make_uint4(0, 0, 0, 0);
-                a0[i][p] = (va && rb < r) ? ldg_stream(Bs + (size_t)ja * r + rb) : z;
-                a1[i][p] = (vc && rb < r) ? ldg_stream(Bs + (size_t)jc * r + rb) : z;
+                a0[i][p] = (va && rb < r_use) ? ldg_stream(Bs + (size_t)ja * r + rb) : z;
+                a1[i][p] = (vc && rb < r_use) ? ldg_stream(Bs + (size_t)jc * r + rb) : z;
               }
               b0[i][0] = (va && row_c0 >= 0) ? __ldg(y0 + (size_t)row_c0 * d_out + ja) : 0.f;
               b0[i][1] = (va && row_c1 >= 0) ? __ldg(y0 + (size_t)row_c1 * d_out + ja) : 0.f;

@@ -56,6 +56,10 @@ struct TcParams {
   const int* slot_tabs[3];
   __nv_bfloat16* ys[3];
   __nv_bfloat16* ys_lo[3];
+  // per-slot adapter rank (nullable: the stored rank) and the function applied to x A^T (MOIN_ACT_*):
+  const int* rank_tabs[3];     // EPI_SHRINK: table of job j (n_jobs = 0: rank_tabs[0])
+  const int* slot_rank;        // EPI_STORE with plan: table of the projection's pool
+  int act;                     // EPI_SHRINK
   const float* inv_norm;       // EPI_ROUTER
   unsigned long long* keys;    // EPI_ROUTER / EPI_ROUTER2: best (similarity, index) key per row
   unsigned long long* keys2;   // EPI_ROUTER2: runner-up key per row
@@ -137,6 +141,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int nkb_main = (p.K + kBK - 1) / kBK;
 
   int job = 0;   // projection of the current tile (EPI_SHRINK with several jobs), set by tile_info
+  int r_use = (EPI == EPI_SHRINK) ? p.N : p.tail_r;   // rank of the current tile's adapter, set by tile_info
   auto tile_info = [&](int tile, int& row0, int& rows, int& n0, int& slot) {
     int tm = tile / tiles_n;
     n0 = (tile - tm * tiles_n) * BN;
@@ -152,6 +157,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int* tab = p.slot_of_expert;
       if (EPI == EPI_SHRINK && p.n_jobs > 0) tab = (job == 0) ? p.slot_tabs[0] : (job == 1) ? p.slot_tabs[1] : p.slot_tabs[2];
       if (e >= 0 && tab) slot = tab[e];
+      if (EPI == EPI_SHRINK || EPI == EPI_STORE) {
+        const int r_full = (EPI == EPI_SHRINK) ? p.N : p.tail_r;
+        const int* rt = (EPI == EPI_STORE) ? p.slot_rank
+                                           : (job == 0 ? p.rank_tabs[0] : job == 1 ? p.rank_tabs[1] : p.rank_tabs[2]);
+        r_use = (slot >= 0 && rt) ? min(rt[slot], r_full) : r_full;
+      }
     } else {
       row0 = tm * kBM;
       rows = min(kBM, p.M - row0);
@@ -218,7 +229,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           int nk16 = (min(kBK, p.K - kb * kBK) + 15) / 16;
           if (kb >= nkb_main) {
             const int j = kb - nkb_main, rb = (j >= nrb) ? j - nrb : j;
-            nk16 = (min(kBK, p.tail_r - rb * kBK) + 15) / 16;
+            nk16 = (min(kBK, r_use - rb * kBK) + 15) / 16;   // columns beyond the adapter's rank: no MMA (<= 0 steps)
           }
           for (int k = 0; k < nk16; ++k)
             tc_mma_bf16(tmem_d, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb > 0 || k > 0) ? 1u : 0u);
@@ -287,6 +298,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               float f[8];
 #pragma unroll
               for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]) * sc;
+              if (EPI == EPI_SHRINK) {   // function between the low-rank matrices; nothing beyond the adapter's rank
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                  f[e] = (n0 + c + j + e < r_use) ? lora_act(__uint_as_float(v[j + e]), p.act) * sc : 0.f;
+              }
               uint4 o;
               o.x = pack_bf16(f[0], f[1]);
               o.y = pack_bf16(f[2], f[3]);
@@ -492,6 +508,8 @@ moin_status launch_tc_shrink_group(HostState* hs, const PlanView& pv, const moin
     if (!st) st = make_map(&bA[j], pools[j]->A, (uint64_t)pools[j]->n_slots * r, d_in, r);   // one slot's rows, no neighbours
     if (st) return st;
     p.slot_tabs[j] = pools[j]->slot_of_expert;
+    p.rank_tabs[j] = pools[j]->slot_rank;
+    p.act = pools[j]->activation;
     p.ys[j] = hbs[j];
     p.ys_lo[j] = hbs[j] + (size_t)T * r;   // low parts follow the high parts in the workspace
   }
@@ -525,6 +543,7 @@ moin_status launch_tc_fused(HostState* hs, const PlanView& pv, const moin_pool* 
   TcParams p = {};
   p.M = T; p.N = d_out; p.K = d_in; p.header = pv.header; p.tile_row0 = pv.tile_row0; p.tile_rows = pv.tile_rows;
   p.tile_expert = pv.tile_expert; p.slot_of_expert = pool->slot_of_expert; p.tail_r = r; p.rows_per_slot = d_out;
+  p.slot_rank = pool->slot_rank;
   p.y = y; p.ldy = d_out; p.scale = 1.f; p.status = hs->status;
   const long tiles = max_tiles_m * ((d_out + bn - 1) / bn);
   if (bn == 256) return launch_cfg<256, EPI_STORE>(hs, ax, bW, ah, al, bB, p, tiles, stream);

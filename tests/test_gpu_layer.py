@@ -6,7 +6,7 @@ import torch
 import moin_inputs as mi
 import oracle
 import paper_2410_09687_b200 as moin
-from gpu_util import DEV, assert_layer_close, gpu_pool, oracle_layer, run_layer
+from gpu_util import compact_pool_for, DEV, assert_layer_close, gpu_pool, oracle_layer, run_layer
 
 pytestmark = pytest.mark.gpu
 MODES = [moin.PLAN_SEGMENTS, moin.PLAN_TILES]
@@ -187,6 +187,60 @@ def test_seeded_random_shapes_in_every_plan_mode(seed):
         for mode in (moin.PLAN_SEGMENTS, moin.PLAN_TILES, moin.PLAN_AUTO):
             y, _ = run_layer(case, mode)
             assert_layer_close(y, ref, f"seed {seed} case {it} mode {mode}: r {r}, {d_in}->{d_out}, E {E}, T {len(te)}")
+
+
+def _variant_case(seed, mode, r, T=300, E=12, d_in=512, d_out=328):
+    rng = mi.np_rng(seed, 1)
+    pool = mi.make_pool(E, r, d_in, d_out, seed, 2, missing=(5,))
+    if mode == moin.PLAN_SEGMENTS:
+        te = rng.integers(-1, E, size=T).astype(np.int32)
+    else:
+        lens = rng.multinomial(T - 6, [1 / 6] * 6) + 1
+        te = np.repeat(rng.integers(0, E, size=6), lens).astype(np.int32)
+    return pool, mi.layer_case("variant", len(te), d_in, d_out, pool, te, 2.0, seed, 3), te
+
+
+@pytest.mark.parametrize("act", [moin.ACT_RELU, moin.ACT_SILU, moin.ACT_GELU])
+@pytest.mark.parametrize("mode", MODES)
+def test_activation_between_the_low_rank_matrices(act, mode):
+    """y = W x + s W_b act(W_a x) (the paper's future-work variant, Sec. 5) against the oracle, both plan modes."""
+    pool, case, te = _variant_case(31, mode, 40)
+    gp = moin.Pool(pool.A.to(DEV), pool.B.to(DEV), pool.slot_of_expert.to(DEV), activation=act)
+    y, _ = run_layer(case, mode, pool=gp)
+    A, B, so = compact_pool_for(pool, te)
+    ref = oracle.lora_linear(mi.bf16_bits(case.x), mi.bf16_bits(case.W), A, B, te, so, case.scale, act=act)
+    assert_layer_close(y, ref, f"activation {act}")
+    plain = oracle.lora_linear(mi.bf16_bits(case.x), mi.bf16_bits(case.W), A, B, te, so, case.scale)
+    assert np.linalg.norm(ref - plain) / np.linalg.norm(plain) > 0.02    # the activation is not a no-op here
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("r", [64, 128])
+def test_mixed_rank_pool(mode, r):
+    """A rank per slot (the paper's future-work "adaptive rank", Sec. 5): pools storing rank r whose slots use
+    8 ... r of it.  What is stored beyond a slot's rank is large finite garbage: it must not reach the result."""
+    pool, case, te = _variant_case(37, mode, r)
+    n_slots = pool.A.shape[0]
+    ranks = np.array([[8, 16, r, 24, r // 2, 0][i % 6] for i in range(n_slots)], np.int32)
+    A, B = pool.A.clone(), pool.B.clone()
+    for s_, k in enumerate(ranks):
+        A[s_, k:, :] = 3.0e38
+        B[s_, :, k:] = -3.0e38
+    gp = moin.Pool(A.to(DEV), B.to(DEV), pool.slot_of_expert.to(DEV), slot_rank=torch.from_numpy(ranks).to(DEV))
+    y, _ = run_layer(case, mode, pool=gp)
+    ref = oracle.lora_linear(mi.bf16_bits(case.x), mi.bf16_bits(case.W), mi.bf16_bits(A), mi.bf16_bits(B), te,
+                             pool.slot_of_expert.numpy(), case.scale, slot_rank=ranks)
+    assert_layer_close(y, ref, f"mixed ranks, stored {r}")
+    # with activation on top, and against the uniform-rank result to see that the ranks matter
+    gp2 = moin.Pool(A.to(DEV), B.to(DEV), pool.slot_of_expert.to(DEV), slot_rank=torch.from_numpy(ranks).to(DEV),
+                    activation=moin.ACT_SILU)
+    y2, _ = run_layer(case, mode, pool=gp2)
+    ref2 = oracle.lora_linear(mi.bf16_bits(case.x), mi.bf16_bits(case.W), mi.bf16_bits(A), mi.bf16_bits(B), te,
+                              pool.slot_of_expert.numpy(), case.scale, slot_rank=ranks, act=oracle.ACT_SILU)
+    assert_layer_close(y2, ref2, f"mixed ranks + SiLU, stored {r}")
+    full = oracle.lora_linear(mi.bf16_bits(case.x), mi.bf16_bits(case.W), mi.bf16_bits(pool.A), mi.bf16_bits(pool.B), te,
+                              pool.slot_of_expert.numpy(), case.scale)
+    assert np.linalg.norm(ref - full) / np.linalg.norm(full) > 0.02
 
 
 def test_empty_batch_and_argument_errors():
