@@ -824,6 +824,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-router-extra", action="store_true")
     ap.add_argument("--no-side-workloads", action="store_true", help="decode line without the prefill / forward keys")
+    ap.add_argument("--print-timeline", action="store_true",
+                    help="also print the kernel timeline of one step (start / end / duration in us) to stderr")
     ap.add_argument("--forward-layers", type=int, default=22)
     ap.add_argument("--no-group", action="store_true", help="one moin_lora_linear call per projection")
     ap.add_argument("--cache-slots", type=int, default=None,
@@ -891,6 +893,11 @@ def main():
     kernels = {k: {"launches": a["launches"], "ms_per_launch": a["ms"] / max(a["launches"], 1)} for k, a in agg.items()}
     tl = kernel_timeline(wl.step, use_graph) if (rank == 0 and kind != "forward" and wl_cache_free(wl)) else None
     path = critical_path(*tl) if tl else None
+    if tl and args.print_timeline:
+        sys.stderr.write("kernel timeline of one step (us from the step's first kernel): start end duration name\n")
+        for name, a, b in tl[0]:
+            sys.stderr.write(f"{a:9.2f} {b:9.2f} {b - a:8.2f}  {name.split('(')[0][:90]}\n")
+        sys.stderr.write(f"step span {tl[1]:.2f} us\n")
     prof_steps = min(args.steps, 20)
     roof = None
     extra = {}
