@@ -364,6 +364,10 @@ typedef struct {
   const void* const* W;          /* host array [n_layers*7] of device [d_out, d_in] bf16; order q,k,v,o,gate,up,down */
   const moin_pool* pools;        /* host array [n_layers*7] or NULL (base model) */
   int32_t E;                     /* expert ids in [0, E) */
+  /* Optional quantised base (see moin_dequant_fp8): host arrays [n_layers*7], either both NULL or both set; where
+   * W8[i] is non-NULL the projection's weight is the dequantised W8[i] / W_scale[i] and W[i] is not read. */
+  const void* const* W8;         /* device [d_out, d_in] bytes */
+  const float* const* W_scale;   /* device [d_out] fp32 */
 } moin_model;
 
 /* Optional taps for block-by-block checks.  hidden_in (nullable, [T, hidden] fp32): start from this
@@ -386,6 +390,21 @@ moin_status moin_decoder_forward(const moin_model* model, const int32_t* tokens,
                                  const int32_t* req_expert, int32_t R, int32_t T, int32_t max_seqlen,
                                  void* logits, int32_t logits_mode, const moin_decoder_taps* taps,
                                  void* workspace, size_t workspace_bytes, moin_stream stream);
+
+/* Quantised frozen base weights with 16-bit adapters.  Paper Sec. 5 lists a quantised base model ("QLoRA-like") as
+ * a variant and fixes no format; the one taken here: one byte per weight in the 8-bit floating-point format with 4
+ * exponent and 3 mantissa bits (bias 7, no infinities, 0x7F / 0xFF = NaN, largest finite value 448) and one fp32
+ * scale per output row.  The weight the layer uses is W[j][i] = bf16(fp32(value(codes[j][i]) * scale[j])): this call
+ * writes it, and the ordinary entry points then run on it, so the adapters, the accumulation and the tolerance are
+ * those of the bf16 layer.  The base model is then stored in half of its bf16 size; a decoder forward with
+ * moin_model.W8 set dequantises one projection group at a time into its workspace (at most three matrices live).
+ *   codes  device, [d_out, d_in] bytes, 16-byte aligned; d_in a multiple of 16
+ *   scale  device, [d_out] fp32
+ *   W      device, [d_out, d_in] bf16, 16-byte aligned (output)
+ * Asynchronous on `stream`.  Errors: MOIN_ERR_INVALID_ARG (null pointer, negative size), MOIN_ERR_BAD_SHAPE,
+ * MOIN_ERR_MISALIGNED. */
+moin_status moin_dequant_fp8(const void* codes, const float* scale, int32_t d_out, int32_t d_in, void* W,
+                             moin_stream stream);
 
 /* The same forward with one expert id per TOKEN: token_expert [T] int32, device, -1 = base only for that token.
  * Paper Sec. 5 (future work: "per-token adapters"); Sec. 3.3 itself uses one expert per request, which is the case

@@ -72,6 +72,10 @@ def lib() -> ctypes.CDLL:
                                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64,
                                                   ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        L.moin_oracle_e4m3_value.restype = ctypes.c_double
+        L.moin_oracle_e4m3_value.argtypes = [ctypes.c_int]
+        L.moin_oracle_dequant_fp8.restype = ctypes.c_int
+        L.moin_oracle_dequant_fp8.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]
         L.moin_oracle_bucket.restype = ctypes.c_int64
         L.moin_oracle_bucket.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                          ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
@@ -173,6 +177,23 @@ def lora_linear(x: np.ndarray, W: np.ndarray, A: Optional[np.ndarray], B: Option
     if rc:
         raise RuntimeError(f"moin_oracle_lora_linear failed: {rc}")
     return y
+
+
+def e4m3_value(code: int) -> float:
+    return float(lib().moin_oracle_e4m3_value(int(code)))
+
+
+def dequant_fp8(codes: np.ndarray, scale: np.ndarray) -> np.ndarray:
+    """bf16 bit patterns [d_out, d_in] of the weight a quantised base layer uses: bf16(fp32(value(code) * scale[row]))."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    scale = np.ascontiguousarray(scale, dtype=np.float32)
+    d_out, d_in = codes.shape
+    assert scale.shape == (d_out,)
+    out = np.zeros((d_out, d_in), np.uint16)
+    rc = lib().moin_oracle_dequant_fp8(_ptr(codes), _ptr(scale), d_out, d_in, _ptr(out))
+    if rc:
+        raise RuntimeError(f"moin_oracle_dequant_fp8 failed: {rc}")
+    return out
 
 
 def bucket(token_expert: np.ndarray, slot_of_expert: np.ndarray, n_slots: int) -> Dict[str, np.ndarray]:

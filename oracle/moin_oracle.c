@@ -509,3 +509,39 @@ int moin_oracle_kmeans_update(const void* x, const void* c_old, int dtype, const
     }
   return 0;
 }
+
+/* ------------------------------------------------------------------------------------
+ * Quantised frozen base weights (Sec. 5 lists a quantised base model with the adapters kept
+ * in 16 bits, "QLoRA-like", as a variant; it fixes no format).  Format taken here: one byte per
+ * weight in the 8-bit floating-point format with 4 exponent and 3 mantissa bits, exponent
+ * bias 7, no infinities (exponent 15 with mantissa 7 is NaN, largest finite value 448), plus
+ * one fp32 scale per output row.  The weight the layer uses is
+ *     W[j][i] = bf16( fp32( value(code[j][i]) * scale[j] ) ),
+ * i.e. the code's value times the row scale, multiplied in fp32 and rounded once more to the
+ * bf16 the GEMMs read.  Everything after that is the ordinary layer on W.
+ * ------------------------------------------------------------------------------------ */
+static float e4m3_value(uint8_t c) {
+  int sign = c >> 7, ex = (c >> 3) & 15, man = c & 7;
+  float v;
+  if (ex == 15 && man == 7) return NAN;
+  if (ex == 0) v = ldexpf((float)man, -9);                 /* subnormal: man / 8 * 2^-6 */
+  else v = ldexpf(1.0f + (float)man / 8.0f, ex - 7);
+  return sign ? -v : v;
+}
+
+double moin_oracle_e4m3_value(int code) { return (double)e4m3_value((uint8_t)code); }
+
+int moin_oracle_dequant_fp8(const uint8_t* codes, const float* scale, int64_t d_out, int64_t d_in,
+                            uint16_t* out_bf16 /* [d_out][d_in] bf16 bit patterns */) {
+  if (!codes || !scale || !out_bf16 || d_out < 0 || d_in < 0) return -1;
+  for (int64_t j = 0; j < d_out; ++j)
+    for (int64_t i = 0; i < d_in; ++i) {
+      volatile float prod = e4m3_value(codes[j * d_in + i]) * scale[j];   /* fp32 product, rounded to fp32 */
+      double r = round_bf16((double)prod);
+      float f = (float)r;                                                  /* exact: r is a bf16 value */
+      uint32_t u;
+      memcpy(&u, &f, 4);
+      out_bf16[j * d_in + i] = (uint16_t)(u >> 16);
+    }
+  return 0;
+}

@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "moin_decoder_workspace_bytes", "moin_decoder_forward", "moin_profile_enable", "moin_profile_read",
     "moin_kernel_name", "moin_route_static", "moin_lora_linear_group", "moin_lora_linear_group_workspace_bytes",
     "moin_kmeans_update", "moin_route_top2", "moin_route_top2_workspace_bytes", "moin_cache_create", "moin_cache_destroy", "moin_cache_admit", "moin_cache_slot_of",
-    "moin_selftest_bounded_wait", "moin_decoder_forward_per_token",
+    "moin_selftest_bounded_wait", "moin_decoder_forward_per_token", "moin_dequant_fp8",
 )
 
 
@@ -63,7 +63,8 @@ class _Model(ctypes.Structure):
                [(n, ctypes.c_float) for n in ("rms_eps", "rope_base", "lora_scale")] + \
                [("embed", ctypes.c_void_p), ("lm_head", ctypes.c_void_p), ("final_norm", ctypes.c_void_p),
                 ("attn_norm", ctypes.POINTER(ctypes.c_void_p)), ("mlp_norm", ctypes.POINTER(ctypes.c_void_p)),
-                ("W", ctypes.POINTER(ctypes.c_void_p)), ("pools", ctypes.POINTER(_Pool)), ("E", ctypes.c_int32)]
+                ("W", ctypes.POINTER(ctypes.c_void_p)), ("pools", ctypes.POINTER(_Pool)), ("E", ctypes.c_int32),
+                ("W8", ctypes.POINTER(ctypes.c_void_p)), ("W_scale", ctypes.POINTER(ctypes.c_void_p))]
 
 
 class _Taps(ctypes.Structure):
@@ -131,6 +132,7 @@ def lib() -> ctypes.CDLL:
         L.moin_decoder_forward.argtypes = [ctypes.POINTER(_Model), vp, vp, vp, i32, i32, i32, vp, i32,
                                            ctypes.POINTER(_Taps), vp, sz, vp]
         L.moin_decoder_forward_per_token.argtypes = L.moin_decoder_forward.argtypes
+        L.moin_dequant_fp8.argtypes = [vp, vp, i32, i32, vp, vp]
         L.moin_profile_enable.argtypes = [i32]
         L.moin_profile_read.argtypes = [ctypes.POINTER(_ProfRec), i32, ctypes.POINTER(i32)]
         L.moin_kernel_name.restype = ctypes.c_char_p
@@ -462,13 +464,15 @@ class DecoderModel:
 
     def __init__(self, cfg, embed, lm_head, final_norm, attn_norm: Sequence[torch.Tensor],
                  mlp_norm: Sequence[torch.Tensor], W: Sequence[dict], pools: Optional[Sequence[dict]], E: int,
-                 lora_scale: float):
+                 lora_scale: float, W8: Optional[Sequence[dict]] = None, W_scale: Optional[Sequence[dict]] = None):
+        """``W8[l][name]`` (uint8 codes) with ``W_scale[l][name]`` (fp32 per output row): quantised base; the entries
+        of ``W`` for those projections may then be None."""
         nl = cfg.n_layers
-        self._keep = [embed, lm_head, final_norm, list(attn_norm), list(mlp_norm), list(W), pools]
+        self._keep = [embed, lm_head, final_norm, list(attn_norm), list(mlp_norm), list(W), pools, W8, W_scale]
         self.cfg = cfg
         self._an = (ctypes.c_void_p * nl)(*[_ptr(t) for t in attn_norm])
         self._mn = (ctypes.c_void_p * nl)(*[_ptr(t) for t in mlp_norm])
-        self._W = (ctypes.c_void_p * (nl * 7))(*[_ptr(W[l][p]) for l in range(nl) for p in PROJ_ORDER])
+        self._W = (ctypes.c_void_p * (nl * 7))(*[_ptr(W[l].get(p)) for l in range(nl) for p in PROJ_ORDER])
         self._pools = None
         if pools is not None:
             self._pools = (_Pool * (nl * 7))(*[pools[l][p].c for l in range(nl) for p in PROJ_ORDER])
@@ -483,6 +487,11 @@ class DecoderModel:
         if self._pools is not None:
             m.pools = ctypes.cast(self._pools, ctypes.POINTER(_Pool))
         m.E = E
+        if W8 is not None:
+            self._W8 = (ctypes.c_void_p * (nl * 7))(*[_ptr(W8[l].get(p)) for l in range(nl) for p in PROJ_ORDER])
+            self._Ws = (ctypes.c_void_p * (nl * 7))(*[_ptr(W_scale[l].get(p)) for l in range(nl) for p in PROJ_ORDER])
+            m.W8 = ctypes.cast(self._W8, ctypes.POINTER(ctypes.c_void_p))
+            m.W_scale = ctypes.cast(self._Ws, ctypes.POINTER(ctypes.c_void_p))
         self.c = m
         self.device = embed.device
         self._ws: Optional[torch.Tensor] = None
@@ -492,6 +501,16 @@ class DecoderModel:
         if self._ws is None or self._ws.numel() < n:
             self._ws = torch.empty(n, dtype=torch.uint8, device=self.device)
         return self._ws
+
+
+def dequant_fp8(codes: torch.Tensor, scale: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """moin_dequant_fp8: uint8 codes [d_out, d_in] and fp32 scale [d_out] -> bf16 weight [d_out, d_in]."""
+    assert codes.dtype == torch.uint8 and scale.dtype == torch.float32 and codes.dim() == 2
+    d_out, d_in = codes.shape
+    if out is None:
+        out = torch.empty(d_out, d_in, dtype=torch.bfloat16, device=codes.device)
+    _check(lib().moin_dequant_fp8(_ptr(codes), _ptr(scale), d_out, d_in, _ptr(out), _stream(stream)), "moin_dequant_fp8")
+    return out
 
 
 def decoder_forward(model: DecoderModel, tokens: torch.Tensor, cu_seqlens: torch.Tensor,

@@ -22,6 +22,34 @@ token_meta_kernel(const int* __restrict__ cu, const int* __restrict__ req_expert
   if (threadIdx.x == 0) last_row[r] = (t1 > t0) ? t1 - 1 : -1;
 }
 
+// W[j][i] = bf16(fp32(value(code[j][i]) * scale[j])): 8-bit float codes (4 exponent bits, bias 7, 3 mantissa bits,
+// no infinities, 0x7F / 0xFF = NaN) -> the bf16 weight the GEMMs read.  One thread converts 16 codes.
+__device__ __forceinline__ float e4m3_to_float(uint32_t c) {
+  const uint32_t sign = (c & 0x80u) << 24, ex = (c >> 3) & 15u, man = c & 7u;
+  if (ex == 15u && man == 7u) return __uint_as_float(0x7FC00000u);
+  if (ex == 0u) return __uint_as_float(sign | __float_as_uint((float)man * 0.001953125f));   // man * 2^-9
+  return __uint_as_float(sign | ((ex + 120u) << 23) | (man << 20));
+}
+__global__ void __launch_bounds__(256)
+dequant_fp8_kernel(const uint4* __restrict__ codes, const float* __restrict__ scale, int d_in16, long n16,
+                   uint4* __restrict__ out) {
+  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n16) return;
+  const float sc = __ldg(scale + i / d_in16);
+  const uint4 c = ldg_stream(codes + i);
+  const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+  uint32_t o[8];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const float f0 = e4m3_to_float(w[k] & 0xFFu) * sc, f1 = e4m3_to_float((w[k] >> 8) & 0xFFu) * sc;
+    const float f2 = e4m3_to_float((w[k] >> 16) & 0xFFu) * sc, f3 = e4m3_to_float(w[k] >> 24) * sc;
+    o[2 * k] = pack_bf16(f0, f1);
+    o[2 * k + 1] = pack_bf16(f2, f3);
+  }
+  out[2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
+  out[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
 // cos/sin of pos * base^(-2i/hd), computed in double once per call.
 __global__ void rope_table_kernel(float2* __restrict__ table, int n_pos, int half, double base) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -295,6 +323,7 @@ attention_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
 
 struct DecoderWorkspace {
   float* res; __nv_bfloat16 *xn, *q, *k, *v, *vt, *att, *o, *gate, *up, *xlast;
+  __nv_bfloat16* wq[3];   // dequantised weights of the projection group in flight (quantised base only)
   int *pos, *token_expert, *last_row;
   float2* rope;
   void* plan; size_t plan_bytes;
@@ -320,6 +349,7 @@ static DecoderWorkspace carve(const moin_model* m, int R, int T, int max_seqlen,
   w.gate = (__nv_bfloat16*)take(TT * F * 2);
   w.up = (__nv_bfloat16*)take(TT * F * 2);
   w.xlast = (__nv_bfloat16*)take((size_t)R * H * 2);
+  for (int i = 0; i < 3; ++i) w.wq[i] = m->W8 ? (__nv_bfloat16*)take(F * (H > qd ? H : qd) * 2) : nullptr;
   w.pos = (int*)take(TT * 4);
   w.token_expert = (int*)take(TT * 4);
   w.last_row = (int*)take((size_t)R * 4 + 4);
@@ -395,8 +425,21 @@ static moin_status decoder_forward_impl(const moin_model* m, const int32_t* toke
     ProfScope prof(MOIN_K_GLUE, 1, s);
     embed_kernel<<<T, 256, 0, s>>>(tokens, (const __nv_bfloat16*)m->embed, H, m->vocab, w.res);
   }
+  // weight of projection p: the caller's bf16 matrix, or - quantised base - its codes dequantised into scratch slot
+  // `slot` on the call's stream (the group calls join their side streams before they return, so a slot is free again)
+  moin_status wst = MOIN_OK;
+  auto weight = [&](int layer, int p, int d_in, int d_out, int slot) -> const void* {
+    const int i = layer * 7 + p;
+    if (!m->W8 || !m->W8[i]) return m->W[i];
+    if (!m->W_scale || !m->W_scale[i]) { wst = MOIN_ERR_INVALID_ARG; return nullptr; }
+    moin_status e = moin_dequant_fp8(m->W8[i], m->W_scale[i], d_out, d_in, w.wq[slot], stream);
+    if (e) wst = e;
+    return w.wq[slot];
+  };
   auto proj = [&](int layer, int p, const void* in, int d_in, int d_out, void* out) -> moin_status {
-    return moin_lora_linear(lora ? &plan : nullptr, in, m->W[layer * 7 + p], lora ? &m->pools[layer * 7 + p] : nullptr,
+    const void* W = weight(layer, p, d_in, d_out, 0);
+    if (wst) return wst;
+    return moin_lora_linear(lora ? &plan : nullptr, in, W, lora ? &m->pools[layer * 7 + p] : nullptr,
                             m->lora_scale, T, d_in, d_out, out, w.lora, w.lora_bytes, stream);
   };
   // projections of a block that read the same input and do not depend on one another go out as one group
@@ -410,7 +453,8 @@ static moin_status decoder_forward_impl(const moin_model* m, const int32_t* toke
       return MOIN_OK;
     }
     moin_lora_job jobs[MOIN_MAX_GROUP];
-    for (int i = 0; i < n; ++i) jobs[i] = {in, m->W[layer * 7 + p0 + i], &m->pools[layer * 7 + p0 + i], outs[i]};
+    for (int i = 0; i < n; ++i) jobs[i] = {in, weight(layer, p0 + i, d_in[i], d_out[i], i), &m->pools[layer * 7 + p0 + i], outs[i]};
+    if (wst) return wst;
     return moin_lora_linear_group(&plan, jobs, n, m->lora_scale, w.lora, w.lora_bytes, stream);
   };
   const float scale_log2 = 1.4426950408889634f / sqrtf(64.f);
@@ -488,4 +532,20 @@ extern "C" moin_status moin_decoder_forward_per_token(const moin_model* m, const
   if (!token_expert) return MOIN_ERR_INVALID_ARG;
   return decoder_forward_impl(m, tokens, cu_seqlens, nullptr, token_expert, R, T, max_seqlen, logits, logits_mode, taps,
                               workspace, workspace_bytes, stream);
+}
+
+extern "C" moin_status moin_dequant_fp8(const void* codes, const float* scale, int32_t d_out, int32_t d_in, void* W,
+                                        moin_stream stream) {
+  if (!codes || !scale || !W || d_out < 0 || d_in < 0) return MOIN_ERR_INVALID_ARG;
+  if ((d_in % 16) != 0) return MOIN_ERR_BAD_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(codes) & 15u) || (reinterpret_cast<uintptr_t>(W) & 15u)) return MOIN_ERR_MISALIGNED;
+  const long n16 = (long)d_out * d_in / 16;
+  if (n16 == 0) return MOIN_OK;
+  HostState* hs;
+  moin_status st = host_state(&hs);
+  if (st) return st;
+  ProfScope prof(MOIN_K_GLUE, 1, (cudaStream_t)stream);
+  dequant_fp8_kernel<<<(unsigned)((n16 + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+      (const uint4*)codes, scale, d_in / 16, n16, (uint4*)W);
+  return record_cuda(cudaGetLastError());
 }

@@ -167,7 +167,9 @@ lora_shrink_stream_kernel(const int* __restrict__ header, const int* __restrict_
 // of adapter bytes, whatever the mix of projection widths in the launch, and a warp's range is contiguous
 // in memory inside a (segment, job).  A warp walks its range kExpandTilesPerBatch tiles at a time with
 // the adapter rows and the base values y0 of a batch loaded together.  `jobs.per_seg[j]` = tiles of job j.
-template <int P>  // number of 32-wide rho groups: ceil(max r / 32)
+// VAR: some pool of the launch has a rank per slot or an activation; without it the kernel is the plain layer's
+// (the rank is the stored rank, h is used as it is) and carries none of the variant's bookkeeping.
+template <int P, bool VAR>  // P: number of 32-wide rho groups, ceil(max r / 32)
 __global__ void __launch_bounds__(kExpandThreads, 4)
 lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict__ perm,
                           const int4* __restrict__ seg_tab, const ExpandJobs jobs, float scale, int tps) {
@@ -191,7 +193,7 @@ lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict_
     int ranks[kMaxStreamJobs];   // rank of the slot's adapter: columns of B and entries of h beyond it are not read
 #pragma unroll
     for (int j = 0; j < kMaxStreamJobs; ++j)
-      ranks[j] = (j < jobs.n && slots[j] >= 0 && jobs.slot_rank[j]) ? min(__ldg(jobs.slot_rank[j] + slots[j]), jobs.r[j])
+      ranks[j] = (VAR && j < jobs.n && slots[j] >= 0 && jobs.slot_rank[j]) ? min(__ldg(jobs.slot_rank[j] + slots[j]), jobs.r[j])
                                                                      : (j < jobs.n ? jobs.r[j] : 0);
     const int row_first = (g < n) ? __ldg(perm + s0 + g) : -1;
     const long long seg_end = (long long)(seg + 1) * tps;
@@ -213,7 +215,7 @@ lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict_
       const int slot = pick(slots, job);
       if (slot >= 0) {
         const int r = pick(jobs.r, job), d_out = pick(jobs.d_out, job);
-        const int r_use = pick(ranks, job), act = pick(jobs.act, job);
+        const int r_use = VAR ? pick(ranks, job) : r, act = VAR ? pick(jobs.act, job) : MOIN_ACT_NONE;
         const float* __restrict__ h = pick(jobs.h, job);
         const float* __restrict__ y0 = pick(jobs.y0, job);
         __nv_bfloat16* __restrict__ y = pick(jobs.y, job);
@@ -237,7 +239,8 @@ lora_expand_stream_kernel(const int* __restrict__ header, const int* __restrict_
             }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              const float s0v = lora_act(v[2 * q], act) * scale, s1v = lora_act(v[2 * q + 1], act) * scale;
+              const float s0v = (VAR ? lora_act(v[2 * q], act) : v[2 * q]) * scale;
+              const float s1v = (VAR ? lora_act(v[2 * q + 1], act) : v[2 * q + 1]) * scale;
               const uint32_t hi = pack_bf16(s0v, s1v);
               hh[p][q] = hi;
               hl[p][q] = pack_bf16(s0v - bf16_lo(hi), s1v - bf16_hi(hi));
@@ -327,12 +330,17 @@ cudaError_t launch_lora_expand_stream(const PlanView& pv, ExpandJobs jobs, float
   // one warp per 2 tiles at least; at most one CTA per resident slot (4 per SM)
   const long max_ctas = ((long)pv.Smax * tps + 2 * (kExpandThreads / 32) - 1) / (2 * (kExpandThreads / 32));
   const int grid = stream_grid(max_ctas, n_sms, 4);
-  if (rmax <= 32)
-    lora_expand_stream_kernel<1><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale, tps);
-  else if (rmax <= 64)
-    lora_expand_stream_kernel<2><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale, tps);
-  else
-    lora_expand_stream_kernel<4><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale, tps);
+  bool var = false;
+  for (int j = 0; j < jobs.n; ++j) var = var || jobs.slot_rank[j] != nullptr || jobs.act[j] != MOIN_ACT_NONE;
+#define MOIN_EXPAND(P)                                                                                          \
+  do {                                                                                                          \
+    if (var) lora_expand_stream_kernel<P, true><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale, tps); \
+    else lora_expand_stream_kernel<P, false><<<grid, kExpandThreads, 0, stream>>>(pv.header, pv.perm, pv.seg_tab, jobs, scale, tps);    \
+  } while (0)
+  if (rmax <= 32) MOIN_EXPAND(1);
+  else if (rmax <= 64) MOIN_EXPAND(2);
+  else MOIN_EXPAND(4);
+#undef MOIN_EXPAND
   return cudaGetLastError();
 }
 
