@@ -431,12 +431,13 @@ static int pick_bn(long tiles_m, int N, int n_sms) {
   }
   return best;
 }
-// Few row tiles (decode): a CTA's duration grows with the bytes it pulls, (128 + BN) * K * 2.  This GEMM runs
-// beside the adapter shrink and the expand waits for both, so take the widest tile (fewest CTAs, least
-// re-reading of x) whose per-CTA bytes stay under a budget that keeps the GEMM the shorter of the two
-// (measured on the decode step: 1.1e6 beats both 0.8e6 and 2.2e6).
+// Few row tiles (decode): a CTA's duration grows with the bytes it pulls, (128 + BN) * K * 2 (an SM receives about
+// 64 bytes per clock).  This GEMM runs beside the adapter shrink and the expand waits for both, so take the widest
+// tile (fewest CTAs, least re-reading of x) whose per-CTA bytes stay under a budget that keeps the GEMM the shorter
+// of the two.  Measured on the decode step's kernel timeline: with 0.8e6 no GEMM outlasts its shrink (the single
+// 2048 -> 2048 projection takes 128 x 64 tiles, 16 us beside a 16 us shrink); 1.1e6 left it exposed by 6 us.
 static int pick_bn_small_m(int N, int K) {
-  const double budget = 1.1e6;
+  const double budget = 0.8e6;
   for (int bn : {256, 128}) {
     if ((128.0 + bn) * K * 2 <= budget && N >= bn) return bn;
   }
