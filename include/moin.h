@@ -90,7 +90,9 @@ moin_status moin_selftest_bounded_wait(int32_t limit_us, int32_t* result, moin_s
 /* Testing/tuning knobs (host-side path selection only; every path computes the same function).
  *   MOIN_OPT_GEMM_IMPL: 0 = automatic, 1 = force the warp-MMA kernels, 2 = force the tcgen05 kernels
  *                       (calls whose shapes the forced kernel cannot take fail with MOIN_ERR_BAD_SHAPE). */
-enum { MOIN_OPT_GEMM_IMPL = 1 };
+/*   MOIN_OPT_NVTX: 1 = every kernel group the library launches is wrapped in an NVTX range named like
+ *   moin_kernel_name() (for timelines of tools that read NVTX); 0 (default) = no ranges. */
+enum { MOIN_OPT_GEMM_IMPL = 1, MOIN_OPT_NVTX = 3 };
 moin_status moin_set_option(int32_t key, int32_t value);
 
 /* Per-kernel timing for benchmarks (no counterpart in the paper).  While enabled, every kernel group the
@@ -390,6 +392,16 @@ moin_status moin_decoder_forward(const moin_model* model, const int32_t* tokens,
                                  const int32_t* req_expert, int32_t R, int32_t T, int32_t max_seqlen,
                                  void* logits, int32_t logits_mode, const moin_decoder_taps* taps,
                                  void* workspace, size_t workspace_bytes, moin_stream stream);
+
+/* Integration of a new or retrained expert into a resident pool.  Paper Sec. 1 / Sec. 5: experts are trained
+ * independently and can be added or replaced one at a time.  Copies A_src [r, d_in] and B_src [d_out, r] (bf16;
+ * device memory, or pinned host memory for a truly asynchronous copy) into slot `slot` of the pool and then maps
+ * `expert` to it (slot_of_expert[expert] = slot), all on `stream`: calls issued later on that stream see the new
+ * adapter, earlier ones the old one.  slot = -1 with NULL sources only unmaps the expert (it then runs on the base
+ * model alone, Sec. 4).  The pool's tensors are the caller's; this call is the one place where the library writes
+ * to them.  Errors: MOIN_ERR_INVALID_ARG (null pool / pointers, expert outside [0, E), slot outside [-1, n_slots)). */
+moin_status moin_pool_set_adapter(const moin_pool* pool, int32_t expert, int32_t slot, const void* A_src,
+                                  const void* B_src, moin_stream stream);
 
 /* Quantised frozen base weights with 16-bit adapters.  Paper Sec. 5 lists a quantised base model ("QLoRA-like") as
  * a variant and fixes no format; the one taken here: one byte per weight in the 8-bit floating-point format with 4

@@ -15,6 +15,7 @@ _lib: Optional[ctypes.CDLL] = None
 PLAN_AUTO, PLAN_SEGMENTS, PLAN_TILES = 0, 1, 2
 LOGITS_ALL, LOGITS_LAST, LOGITS_NONE = 0, 1, 2
 OPT_GEMM_IMPL = 1
+OPT_NVTX = 3
 ACT_NONE, ACT_RELU, ACT_SILU, ACT_GELU = 0, 1, 2, 3
 
 EXPORTED_SYMBOLS = (
@@ -24,7 +25,7 @@ EXPORTED_SYMBOLS = (
     "moin_decoder_workspace_bytes", "moin_decoder_forward", "moin_profile_enable", "moin_profile_read",
     "moin_kernel_name", "moin_route_static", "moin_lora_linear_group", "moin_lora_linear_group_workspace_bytes",
     "moin_kmeans_update", "moin_route_top2", "moin_route_top2_workspace_bytes", "moin_cache_create", "moin_cache_destroy", "moin_cache_admit", "moin_cache_slot_of",
-    "moin_selftest_bounded_wait", "moin_decoder_forward_per_token", "moin_dequant_fp8",
+    "moin_selftest_bounded_wait", "moin_decoder_forward_per_token", "moin_dequant_fp8", "moin_pool_set_adapter",
 )
 
 
@@ -133,6 +134,7 @@ def lib() -> ctypes.CDLL:
                                            ctypes.POINTER(_Taps), vp, sz, vp]
         L.moin_decoder_forward_per_token.argtypes = L.moin_decoder_forward.argtypes
         L.moin_dequant_fp8.argtypes = [vp, vp, i32, i32, vp, vp]
+        L.moin_pool_set_adapter.argtypes = [ctypes.POINTER(_Pool), i32, i32, vp, vp, vp]
         L.moin_profile_enable.argtypes = [i32]
         L.moin_profile_read.argtypes = [ctypes.POINTER(_ProfRec), i32, ctypes.POINTER(i32)]
         L.moin_kernel_name.restype = ctypes.c_char_p
@@ -350,6 +352,18 @@ class Pool:
         self.E, self.n_slots, self.r, self.d_in, self.d_out = slot_of_expert.shape[0], n_slots, r, d_in, d_out
         self.c = _Pool(_ptr(A), _ptr(B), _ptr(slot_of_expert), self.E, n_slots, r, d_in, d_out, int(activation),
                        _ptr(slot_rank))
+
+
+def pool_set_adapter(pool: Pool, expert: int, slot: int, A: Optional[torch.Tensor] = None,
+                     B: Optional[torch.Tensor] = None, stream=None) -> None:
+    """moin_pool_set_adapter: write one adapter (A [r, d_in], B [d_out, r], device or pinned host) into ``slot`` and
+    map ``expert`` to it; slot = -1 unmaps the expert."""
+    for t in (A, B):
+        assert t is None or (t.dtype == torch.bfloat16 and t.is_contiguous() and (t.is_cuda or t.is_pinned()))
+    pa = None if A is None else A.data_ptr()
+    pb = None if B is None else B.data_ptr()
+    _check(lib().moin_pool_set_adapter(ctypes.byref(pool.c), int(expert), int(slot), pa, pb, _stream(stream)),
+           "moin_pool_set_adapter")
 
 
 class Plan:

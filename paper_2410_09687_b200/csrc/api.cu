@@ -1,6 +1,8 @@
 // C ABI entry points: argument validation, workspace carving, kernel launches.
 #include <string.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 #include "tc_gemm.cuh"
 
@@ -10,7 +12,7 @@ __device__ DeviceStatus g_device_status;
 
 static thread_local int t_last_cuda_error = 0;
 static HostState g_states[kMaxDevices];
-static int g_opt_gemm_impl = 0;   // moin_set_option: process-wide
+static int g_opt_gemm_impl = 0, g_opt_nvtx = 0;   // moin_set_option: process-wide
 
 moin_status record_cuda(cudaError_t e) {
   if (e == cudaSuccess) return MOIN_OK;
@@ -59,7 +61,8 @@ struct ProfState {
 };
 static ProfState g_prof;
 
-ProfScope::ProfScope(int kernel, int launches, cudaStream_t s) : slot(-1), stream(s) {
+ProfScope::ProfScope(int kernel, int launches, cudaStream_t s) : slot(-1), stream(s), nvtx(g_opt_nvtx != 0) {
+  if (nvtx) nvtxRangePushA(moin_kernel_name(kernel));
   if (g_prof.capacity > 0 && g_prof.count < g_prof.capacity) {
     slot = g_prof.count++;
     g_prof.kernel[slot] = kernel;
@@ -69,7 +72,10 @@ ProfScope::ProfScope(int kernel, int launches, cudaStream_t s) : slot(-1), strea
 }
 ProfScope::~ProfScope() {
   if (slot >= 0) cudaEventRecord(g_prof.stop[slot], stream);
+  if (nvtx) nvtxRangePop();
 }
+
+__global__ void set_int_kernel(int* p, int v) { *p = v; }
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -102,7 +108,32 @@ moin_status moin_set_option(int32_t key, int32_t value) {
     g_opt_gemm_impl = value;
     return MOIN_OK;
   }
+  if (key == MOIN_OPT_NVTX && (value == 0 || value == 1)) {
+    g_opt_nvtx = value;
+    return MOIN_OK;
+  }
   return MOIN_ERR_INVALID_ARG;
+}
+
+moin_status moin_pool_set_adapter(const moin_pool* pool, int32_t expert, int32_t slot, const void* A_src,
+                                  const void* B_src, moin_stream stream) {
+  if (!pool || !pool->slot_of_expert || expert < 0 || expert >= pool->E || slot < -1 || slot >= pool->n_slots)
+    return MOIN_ERR_INVALID_ARG;
+  if (slot >= 0 && (!A_src || !B_src || !pool->A || !pool->B)) return MOIN_ERR_INVALID_ARG;
+  HostState* hs;
+  moin_status st = host_state(&hs);
+  if (st) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (slot >= 0) {
+    const size_t na = (size_t)pool->r * pool->d_in * sizeof(__nv_bfloat16), nb = (size_t)pool->d_out * pool->r * sizeof(__nv_bfloat16);
+    char* A = const_cast<char*>(reinterpret_cast<const char*>(pool->A)) + (size_t)slot * na;
+    char* B = const_cast<char*>(reinterpret_cast<const char*>(pool->B)) + (size_t)slot * nb;
+    cudaError_t e = cudaMemcpyAsync(A, A_src, na, cudaMemcpyDefault, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(B, B_src, nb, cudaMemcpyDefault, s);
+    if (e != cudaSuccess) return record_cuda(e);
+  }
+  set_int_kernel<<<1, 1, 0, s>>>(const_cast<int*>(pool->slot_of_expert) + expert, slot);   // after the copies, in stream order
+  return record_cuda(cudaGetLastError());
 }
 
 moin_status moin_device_status(moin_device_status_t* out, moin_stream stream) {

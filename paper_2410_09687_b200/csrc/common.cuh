@@ -208,6 +208,7 @@ struct ProfScope {
   ~ProfScope();
   int slot;
   cudaStream_t stream;
+  bool nvtx;
 };
 
 }  // namespace moin
