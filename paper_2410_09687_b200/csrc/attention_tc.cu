@@ -4,8 +4,9 @@
 // that share a kv head are stacked into one 128-row tile: row r holds position q0 + r / g of head kvh * g + r % g,
 // so a block covers 128 / g positions and every staged K / V tile serves all g heads.  Persistent CTAs (two per
 // SM) walk the items, longest first.  Warp roles:
-//   warp 0      TMA producer: K tiles [64 keys x 64 dims] and V^T tiles [64 dims x 64 keys] into small rings
-//               (V^T comes from a transposed copy of v, so both are K-major operands of the same form the GEMMs use)
+//   warp 0      TMA producer: K and V tiles [64 keys x 64 dims] into small rings.  K is a K-major operand of the
+//               form the GEMMs use; V, whose rows run along the output dimension of the second product, is read
+//               as an MN-major operand (same staged bytes, the other operand layout), so no transposed copy exists
 //   warp 1      MMA issuer: S = Q K^T into one of two TMEM buffers, O += P V into a third
 //   warps 2-9   two threads per tile row (32 of a tile's 64 columns each): rotate and stage Q (128-byte swizzled
 //               rows, written by hand), softmax, P as the bf16 A operand of the second product (swizzled rows
@@ -13,9 +14,8 @@
 // The softmax takes two passes over the keys: the first only finds each row's maximum, the second forms
 // p = 2^(s - max) once per element, sums it in fp32 and multiplies by V - so the O accumulator in TMEM never
 // needs rescaling.  S is recomputed in the second pass (the MMAs are a small part of the time; the
-// exponentials are not).  Key tiles are aligned to multiples of 8 TOKENS of the packed batch (a TMA copy must
-// start on a 16-byte boundary of V^T's rows), so a request's first tile may begin with keys of the request
-// before it: the mask is t0 <= key <= query position, in batch coordinates.
+// exponentials are not).  Key tiles start at the request's first token (only the innermost coordinate of a TMA
+// copy has an alignment rule, and that is the head's first dimension); the mask is key <= query position.
 // Every mbarrier wait is bounded; on expiry the CTA raises the status flag, drains and returns.
 #include <cuda.h>
 
@@ -27,7 +27,7 @@ namespace moin {
 constexpr int kAtThreads = 320;                  // producer warp, MMA warp, 8 softmax warps
 constexpr int kAtKeys = 64;                      // keys per tile
 constexpr int kAtTile = 128 * 64 * 2;            // Q and P tiles: 128 rows x 128 bytes
-constexpr int kAtKV = kAtKeys * 64 * 2;          // K and V^T tiles: 64 rows x 128 bytes
+constexpr int kAtKV = kAtKeys * 64 * 2;          // K and V tiles: 64 keys x 128 bytes
 constexpr int kAtKS = 4, kAtVS = 3;              // ring depths: a tile's loads take about as long as two tiles' work
 constexpr int kAtSmem = kAtTile /*Q*/ + 2 * kAtTile /*P*/ + kAtKS * kAtKV + kAtVS * kAtKV + 1024 /*align*/ +
                         256 /*barriers*/ + 2048 /*row maxima and sums of the two half rows*/;
@@ -55,6 +55,10 @@ __device__ __forceinline__ uint64_t at_sdesc(uint32_t saddr) {
 }
 // D fp32, A / B bf16 K-major, M = 128, N = 64
 constexpr uint32_t kAtIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+// the same with B MN-major (V tile: one 128-byte row per key, the 64 output dims contiguous); a 16-key step of
+// such a tile is two 8-key groups = 2048 bytes further on
+constexpr uint32_t kAtIdescPV = kAtIdesc | (1u << 16);
+constexpr uint64_t kAtVStep = 2048 >> 4;
 
 __device__ __forceinline__ float fast_exp2(float x) {   // arguments are <= 0 here: 2^x in (0, 1]
   float y;
@@ -79,14 +83,14 @@ __device__ __forceinline__ AttItem at_item(const AttParams& p, int idx) {
   it.t0 = __ldg(p.cu + it.req);
   it.L = __ldg(p.cu + it.req + 1) - it.t0;
   it.on = it.q0 < it.L;
-  it.a0 = it.t0 & ~7;
+  it.a0 = it.t0;
   const int kv_end = min(it.L, it.q0 + p.ppt);   // keys of the request this block can see
   it.n_tiles = it.on ? (it.t0 + kv_end - it.a0 + kAtKeys - 1) / kAtKeys : 0;
   return it;
 }
 
 __global__ void __launch_bounds__(kAtThreads, 2)
-attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVt, const AttParams p) {
+attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -149,7 +153,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
               const uint32_t s = vq % kAtVS, ph = (vq / kAtVS) & 1u;
               if (!(ok = mbar_wait(vempty + 8 * s, ph ^ 1u, abort_flag, p.status, 32))) break;
               mbar_expect_tx(vfull + 8 * s, kAtKV);
-              tma_load_2d(sV + s * kAtKV, &tmVt, vfull + 8 * s, a, it.kvh * 64);
+              tma_load_2d(sV + s * kAtKV, &tmV, vfull + 8 * s, it.kvh * 64, a);
               ++vq;
             }
           }
@@ -195,7 +199,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           const uint64_t dp = at_sdesc(sP + b * kAtTile), dv = at_sdesc(sV + s * kAtKV);
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            tc_mma_bf16(tmem + 128, dp + (uint64_t)(2 * k), dv + (uint64_t)(2 * k), kAtIdesc, (j > 0 || k > 0) ? 1u : 0u);
+            tc_mma_bf16(tmem + 128, dp + (uint64_t)(2 * k), dv + kAtVStep * k, kAtIdescPV, (j > 0 || k > 0) ? 1u : 0u);
           tc_commit(vempty + 8 * s);
           tc_commit(pfree + 8 * b);
           ++pq; ++vq;
@@ -367,56 +371,26 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   }
 }
 
-// vt[c][t] = v[t][c]: the second product needs V with the keys contiguous.  Columns T .. Tp of vt are zeroed
-// (they are multiplied by zero weights, which garbage bits might not survive).
-__global__ void __launch_bounds__(256)
-transpose_v_kernel(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ vt, int T, int Tp, int kvd) {
-  __shared__ uint16_t tile[32][33];
-  const int t0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
-  const uint16_t* src = reinterpret_cast<const uint16_t*>(v);
-  uint16_t* dst = reinterpret_cast<uint16_t*>(vt);
-  for (int i = ty; i < 32; i += 8) {
-    const int t = t0 + i, c = c0 + tx;
-    tile[i][tx] = (t < T && c < kvd) ? src[(size_t)t * kvd + c] : (uint16_t)0;
-  }
-  __syncthreads();
-  for (int i = ty; i < 32; i += 8) {
-    const int c = c0 + i, t = t0 + tx;
-    if (c < kvd && t < Tp) dst[(size_t)c * Tp + t] = tile[tx][i];
-  }
-}
-
 bool attention_tc_supported(int n_heads, int n_kv_heads, int head_dim) {
   if (head_dim != 64 || n_kv_heads < 1 || (n_heads % n_kv_heads) != 0) return false;
   const int g = n_heads / n_kv_heads;
   return g >= 1 && g <= 128 && (128 % g) == 0;
 }
 
-size_t attention_tc_scratch_bytes(int T, int n_kv_heads) {
-  const size_t Tp = ((size_t)T + 7) / 8 * 8;
-  return (size_t)n_kv_heads * 64 * Tp * sizeof(__nv_bfloat16);
-}
-
 // q [T, n_heads*64] (not rotated), k [T, n_kv*64] (rotated), v [T, n_kv*64] -> out [T, n_heads*64].
-// vt_scratch: attention_tc_scratch_bytes(T, n_kv) bytes, 256-byte aligned.
 moin_status launch_attention_tc(HostState* hs, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                                const int* cu, __nv_bfloat16* out, __nv_bfloat16* vt_scratch, const float2* rope, int R,
+                                const int* cu, __nv_bfloat16* out, const float2* rope, int R,
                                 int T, int max_seqlen, int n_heads, int n_kv_heads, float scale_log2,
                                 cudaStream_t stream) {
   const int kvd = n_kv_heads * 64, g = n_heads / n_kv_heads;
-  const int Tp = (T + 7) / 8 * 8;
-  transpose_v_kernel<<<dim3((Tp + 31) / 32, (kvd + 31) / 32), 256, 0, stream>>>(v, vt_scratch, T, Tp, kvd);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return record_cuda(e);
   CUtensorMap mk, mv;
   moin_status st = make_map(&mk, k, (uint64_t)T, (uint64_t)kvd, kAtKeys);
-  if (!st) st = make_map(&mv, vt_scratch, (uint64_t)kvd, (uint64_t)Tp, 64);
+  if (!st) st = make_map(&mv, v, (uint64_t)T, (uint64_t)kvd, kAtKeys);
   if (st) return st;
   AttParams p = {};
   p.q = q; p.out = out; p.cu = cu; p.rope = rope; p.R = R; p.n_heads = n_heads; p.n_kv = n_kv_heads; p.g = g;
   p.ppt = 128 / g; p.n_qb = (max_seqlen + p.ppt - 1) / p.ppt; p.scale_log2 = scale_log2; p.status = hs->status;
-  e = ensure_smem_optin(OPTIN_ATTENTION, attention_tc_kernel, kAtSmem);
+  cudaError_t e = ensure_smem_optin(OPTIN_ATTENTION, attention_tc_kernel, kAtSmem);
   if (e != cudaSuccess) return record_cuda(e);
   const long items = (long)p.n_qb * R * n_kv_heads;
   long grid = items < 2L * hs->n_sms ? items : 2L * hs->n_sms;

@@ -322,7 +322,7 @@ attention_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __res
 }
 
 struct DecoderWorkspace {
-  float* res; __nv_bfloat16 *xn, *q, *k, *v, *vt, *att, *o, *gate, *up, *xlast;
+  float* res; __nv_bfloat16 *xn, *q, *k, *v, *att, *o, *gate, *up, *xlast;
   __nv_bfloat16* wq[3];   // dequantised weights of the projection group in flight (quantised base only)
   int *pos, *token_expert, *last_row;
   float2* rope;
@@ -343,7 +343,6 @@ static DecoderWorkspace carve(const moin_model* m, int R, int T, int max_seqlen,
   w.q = (__nv_bfloat16*)take(TT * qd * 2);
   w.k = (__nv_bfloat16*)take(TT * kvd * 2);
   w.v = (__nv_bfloat16*)take(TT * kvd * 2);
-  w.vt = (__nv_bfloat16*)take(attention_tc_scratch_bytes(T, m->n_kv_heads));   // transposed copy of v
   w.att = (__nv_bfloat16*)take(TT * qd * 2);
   w.o = (__nv_bfloat16*)take(TT * H * 2);
   w.gate = (__nv_bfloat16*)take(TT * F * 2);
@@ -471,9 +470,9 @@ static moin_status decoder_forward_impl(const moin_model* m, const int32_t* toke
     // the queries are rotated inside the attention kernel as it loads them
     { ProfScope prof(MOIN_K_GLUE, 1, s);
       rope_kernel<<<(int)(((long)T * nkv * 32 + 255) / 256), 256, 0, s>>>(w.k, w.pos, w.rope, T, nkv); }
-    if (hs->gemm_impl != 1 && attention_tc_supported(nh, nkv, m->head_dim)) {   // tcgen05 kernel (+ transpose of v)
+    if (hs->gemm_impl != 1 && attention_tc_supported(nh, nkv, m->head_dim)) {   // tcgen05 kernel
       ProfScope prof(MOIN_K_ATTENTION, 2, s);
-      if ((st = launch_attention_tc(hs, w.q, w.k, w.v, cu_seqlens, w.att, w.vt, w.rope, R, T, max_seqlen, nh, nkv,
+      if ((st = launch_attention_tc(hs, w.q, w.k, w.v, cu_seqlens, w.att, w.rope, R, T, max_seqlen, nh, nkv,
                                     scale_log2, s)))
         return st;
     } else {   // warp-MMA kernel: other head groupings, or forced by MOIN_OPT_GEMM_IMPL = 1

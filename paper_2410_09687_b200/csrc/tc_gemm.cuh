@@ -32,11 +32,10 @@ constexpr int kTcMaxShrinkJobs = 3;   // projections one grouped shrink launch c
 moin_status launch_tc_fused(HostState* hs, const PlanView& pv, const moin_pool* pool, const __nv_bfloat16* x,
                             const __nv_bfloat16* W, __nv_bfloat16* y, __nv_bfloat16* hb, cudaStream_t stream);
 
-// Causal GQA attention on tcgen05 (attention_tc.cu).  q not rotated, k rotated; vt_scratch holds a transposed copy of v.
+// Causal GQA attention on tcgen05 (attention_tc.cu).  q not rotated, k rotated.
 bool attention_tc_supported(int n_heads, int n_kv_heads, int head_dim);
-size_t attention_tc_scratch_bytes(int T, int n_kv_heads);
 moin_status launch_attention_tc(HostState* hs, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                                const int* cu, __nv_bfloat16* out, __nv_bfloat16* vt_scratch, const float2* rope, int R,
+                                const int* cu, __nv_bfloat16* out, const float2* rope, int R,
                                 int T, int max_seqlen, int n_heads, int n_kv_heads, float scale_log2,
                                 cudaStream_t stream);
 
