@@ -50,7 +50,8 @@ def setup():
 
 
 @pytest.mark.parametrize("lengths,experts", [([70, 1, 129, 33, 64], [0, 2, 3, -1, 5]),      # short requests: segments
-                                             ([200, 130, 257], [1, 1, 4])])                 # long runs: tiles
+                                             ([200, 130, 257], [1, 1, 4]),                  # long runs: tiles
+                                             ([3, 530, 260], [5, 2, 0])])     # attention items beyond 256 keys
 def test_decoder_end_to_end_and_block_by_block(setup, lengths, experts):
     model, gm, orc = setup
     batch = mi.decoder_batch(CFG, lengths, seed=4, req_expert=experts)
