@@ -399,27 +399,85 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       const bool live = pos < it.L;
       uint4 cn[4];
       if (have_nx && it.n_tiles <= kAtResident) q_load(nx, cn);
-      const int lim = it.t0 + pos;               // last visible key, batch coordinates
       const bool resident = it.n_tiles <= kAtResident;
-      // one half tile of scores: row maximum over the visible keys / p = 2^(s - max) as bf16 pairs and their sum
-      auto tile_max = [&](const uint32_t (&v)[32], int key0, float m) -> float {
-        if (key0 + 31 <= lim) {                  // every key of this half tile is visible to this row
+      // Scores come in half tiles of 32 keys, taken as two groups of 16.  Keys are counted from the request's first
+      // token (kr); row `pos` sees kr <= pos.  A group is visible to every row of the item when it ends before the
+      // item's first position, to none when it starts after the item's last one (both the same for all threads:
+      // no exponentials are spent there), and is masked key by key otherwise.
+      const int q_last = it.q0 + p.ppt - 1;
+      auto tile_max = [&](const uint32_t (&v)[32], int kr0, float m) -> float {
 #pragma unroll
-          for (int c = 0; c < 32; c += 2) m = max3(m, __uint_as_float(v[c]), __uint_as_float(v[c + 1]));
-        } else {
+        for (int q = 0; q < 2; ++q) {
+          const int kr = kr0 + 16 * q;
+          if (kr + 15 <= it.q0) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (key0 + c <= lim) m = fmaxf(m, __uint_as_float(v[c]));
+            for (int c = 16 * q; c < 16 * q + 16; c += 2) m = max3(m, __uint_as_float(v[c]), __uint_as_float(v[c + 1]));
+          } else if (kr <= q_last) {
+#pragma unroll
+            for (int c = 16 * q; c < 16 * q + 16; ++c)
+              if (kr0 + c <= pos) m = fmaxf(m, __uint_as_float(v[c]));
+          }
         }
         return m;
       };
-      auto tile_p = [&](const uint32_t (&v)[32], int key0, float mb, uint8_t* prow, float l) -> float {
+      auto tile_p = [&](const uint32_t (&v)[32], int kr0, float mb, uint8_t* prow, float l) -> float {
         uint32_t w[16];
         const uint64_t scale2 = pair_f32(p.scale_log2, p.scale_log2), nmb2 = pair_f32(-mb, -mb);
-        if (key0 + 31 <= lim) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int kr = kr0 + 16 * q;
+          if (kr + 15 <= it.q0) {
+            uint64_t l2 = pair_f32(l, 0.f);
+#pragma unroll
+            for (int c = 16 * q; c < 16 * q + 16; c += 2) {
+              float x0, x1;
+              unpair_f32(fma2(pair_f32(__uint_as_float(v[c]), __uint_as_float(v[c + 1])), scale2, nmb2), x0, x1);
+              const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+              l2 = add2(l2, pair_f32(p0, p1));
+              w[c >> 1] = pack_bf16(p0, p1);
+            }
+            float la, lb;
+            unpair_f32(l2, la, lb);
+            l = la + lb;
+          } else if (kr <= q_last) {
+#pragma unroll
+            for (int c = 16 * q; c < 16 * q + 16; c += 2) {
+              const int k0 = kr0 + c;
+              const float p0 = k0 <= pos ? fast_exp2(fmaf(__uint_as_float(v[c]), p.scale_log2, -mb)) : 0.f;
+              const float p1 = k0 + 1 <= pos ? fast_exp2(fmaf(__uint_as_float(v[c + 1]), p.scale_log2, -mb)) : 0.f;
+              l += p0 + p1;
+              w[c >> 1] = pack_bf16(p0, p1);
+            }
+          } else {
+#pragma unroll
+            for (int c = 16 * q; c < 16 * q + 16; c += 2) w[c >> 1] = 0u;
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)               // chunks 4 half .. 4 half + 3 of this row
+          *reinterpret_cast<uint4*>(prow + at_swz(row, 4 * half + i)) = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+        return l;
+      };
+      // the same for one group of 16 keys at a time (resident items: the TMEM read of the next group is in flight
+      // while this one is worked on); two running maxima keep the dependent chain short
+      auto group_max = [&](const uint32_t (&v)[16], int kr, float& m0, float& m1) {
+        if (kr + 15 <= it.q0) {
+#pragma unroll
+          for (int c = 0; c < 16; c += 4) {
+            m0 = max3(m0, __uint_as_float(v[c]), __uint_as_float(v[c + 1]));
+            m1 = max3(m1, __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
+          }
+        } else if (kr <= q_last) {
+#pragma unroll
+          for (int c = 0; c < 16; ++c)
+            if (kr + c <= pos) m0 = fmaxf(m0, __uint_as_float(v[c]));
+        }
+      };
+      auto group_p = [&](const uint32_t (&v)[16], int kr, uint64_t scale2, uint64_t nmb2, float mb, uint32_t* w, float& l) {
+        if (kr + 15 <= it.q0) {
           uint64_t l2 = pair_f32(l, 0.f);
 #pragma unroll
-          for (int c = 0; c < 32; c += 2) {
+          for (int c = 0; c < 16; c += 2) {
             float x0, x1;
             unpair_f32(fma2(pair_f32(__uint_as_float(v[c]), __uint_as_float(v[c + 1])), scale2, nmb2), x0, x1);
             const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
@@ -429,32 +487,41 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           float la, lb;
           unpair_f32(l2, la, lb);
           l = la + lb;
-        } else {
+        } else if (kr <= q_last) {
 #pragma unroll
-          for (int c = 0; c < 32; c += 2) {
-            const int key = key0 + c;
-            const float p0 = key <= lim ? fast_exp2(fmaf(__uint_as_float(v[c]), p.scale_log2, -mb)) : 0.f;
-            const float p1 = key + 1 <= lim ? fast_exp2(fmaf(__uint_as_float(v[c + 1]), p.scale_log2, -mb)) : 0.f;
+          for (int c = 0; c < 16; c += 2) {
+            const float p0 = kr + c <= pos ? fast_exp2(fmaf(__uint_as_float(v[c]), p.scale_log2, -mb)) : 0.f;
+            const float p1 = kr + c + 1 <= pos ? fast_exp2(fmaf(__uint_as_float(v[c + 1]), p.scale_log2, -mb)) : 0.f;
             l += p0 + p1;
             w[c >> 1] = pack_bf16(p0, p1);
           }
-        }
+        } else {
 #pragma unroll
-        for (int i = 0; i < 4; ++i)               // chunks 4 half .. 4 half + 3 of this row
-          *reinterpret_cast<uint4*>(prow + at_swz(row, 4 * half + i)) = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-        return l;
+          for (int c = 0; c < 8; ++c) w[c] = 0u;
+        }
       };
+      // group g of this thread: tile g / 2, columns half * 32 + 16 (g % 2) of it
+      const uint32_t tcol = tmem + lane_addr + half * 32;
+      auto g_col = [&](int g) -> uint32_t { return tcol + (uint32_t)((g >> 1) * 64 + (g & 1) * 16); };
+      auto g_kr = [&](int g) -> int { return (g >> 1) * kAtKeys + half * 32 + (g & 1) * 16; };
       // ---- pass 1: row maximum of the raw scores (the scale is positive: it commutes with the maximum)
       float m = -INFINITY;
       if (resident) {
         if ((ok = ok && mbar_wait(sall, nres & 1u, abort_flag, p.status, 43))) {
           tc_fence_after();
-          for (int j = 0; j < it.n_tiles; ++j) {
-            uint32_t v[32];
-            tmem_ld32(tmem + lane_addr + j * 64 + half * 32, v);
+          float m1 = -INFINITY;
+          uint32_t va[16], vb[16];
+          const int G = 2 * it.n_tiles;
+          tmem_ld16(g_col(0), va);
+          for (int g = 0; g < G; g += 2) {
             tmem_ld_wait();
-            m = tile_max(v, it.a0 + j * kAtKeys + half * 32, m);
+            tmem_ld16(g_col(g + 1), vb);
+            group_max(va, g_kr(g), m, m1);
+            tmem_ld_wait();
+            if (g + 2 < G) tmem_ld16(g_col(g + 2), va);
+            group_max(vb, g_kr(g + 1), m, m1);
           }
+          m = fmaxf(m, m1);
         }
         ++nres;
       } else {
@@ -465,7 +532,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           uint32_t v[32];
           tmem_ld32(tmem + lane_addr + b * 64 + half * 32, v);
           tmem_ld_wait();
-          m = tile_max(v, it.a0 + j * kAtKeys + half * 32, m);
+          m = tile_max(v, j * kAtKeys + half * 32, m);
           tc_fence_before();
           mbar_arrive(sfree + 8 * b);
           ++sq;
@@ -478,7 +545,32 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       if (have_nx && resident) q_stage(nx, cn);   // every score MMA of this item is complete: the Q tile is free
       // ---- pass 2: p = 2^(s - max), row sum in fp32, P tile as bf16 operand
       float l = 0.f;
-      for (int j = 0; j < it.n_tiles && ok; ++j) {
+      if (resident && ok) {
+        const uint64_t scale2 = pair_f32(p.scale_log2, p.scale_log2), nmb2 = pair_f32(-mb, -mb);
+        uint32_t va[16], vb[16];
+        tmem_ld16(g_col(0), va);
+        for (int j = 0; j < it.n_tiles; ++j) {
+          const uint32_t pb = pq & 1u, pph = (pq >> 1) & 1u;
+          uint32_t w[16];
+          tmem_ld_wait();
+          tmem_ld16(g_col(2 * j + 1), vb);
+          group_p(va, g_kr(2 * j), scale2, nmb2, mb, w, l);
+          tmem_ld_wait();
+          if (j + 1 < it.n_tiles) tmem_ld16(g_col(2 * j + 2), va);
+          group_p(vb, g_kr(2 * j + 1), scale2, nmb2, mb, w + 8, l);
+          if (!(ok = mbar_wait(pfree + 8 * pb, pph ^ 1u, abort_flag, p.status, 41))) break;
+          uint8_t* prow = base_ptr + (sP - base) + pb * kAtTile;
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            *reinterpret_cast<uint4*>(prow + at_swz(row, 4 * half + i)) = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+          tc_fence_before();                      // this tile's scores are read: the O columns over them may be written
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          mbar_arrive(pready + 8 * pb);
+          ++pq;
+        }
+        if (!ok) tmem_ld_wait();
+      }
+      for (int j = 0; j < it.n_tiles && ok && !resident; ++j) {
         const uint32_t b = sq & 1u, bph = (sq >> 1) & 1u, pb = pq & 1u, pph = (pq >> 1) & 1u;
         if (!resident && !(ok = mbar_wait(sready + 8 * b, bph, abort_flag, p.status, 40))) break;
         if (!(ok = mbar_wait(pfree + 8 * pb, pph ^ 1u, abort_flag, p.status, 41))) break;
@@ -486,7 +578,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         uint32_t v[32];
         tmem_ld32(tmem + lane_addr + (resident ? j : (int)b) * 64 + half * 32, v);
         tmem_ld_wait();
-        l = tile_p(v, it.a0 + j * kAtKeys + half * 32, mb, base_ptr + (sP - base) + pb * kAtTile, l);
+        l = tile_p(v, j * kAtKeys + half * 32, mb, base_ptr + (sP - base) + pb * kAtTile, l);
         tc_fence_before();                        // the scores are read: the buffer (resident: the O columns) may be written
         if (!resident) { mbar_arrive(sfree + 8 * b); ++sq; }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -471,7 +471,7 @@ static moin_status decoder_forward_impl(const moin_model* m, const int32_t* toke
     { ProfScope prof(MOIN_K_GLUE, 1, s);
       rope_kernel<<<(int)(((long)T * nkv * 32 + 255) / 256), 256, 0, s>>>(w.k, w.pos, w.rope, T, nkv); }
     if (hs->gemm_impl != 1 && attention_tc_supported(nh, nkv, m->head_dim)) {   // tcgen05 kernel
-      ProfScope prof(MOIN_K_ATTENTION, 2, s);
+      ProfScope prof(MOIN_K_ATTENTION, 1, s);
       if ((st = launch_attention_tc(hs, w.q, w.k, w.v, cu_seqlens, w.att, w.rope, R, T, max_seqlen, nh, nkv,
                                     scale_log2, s)))
         return st;
