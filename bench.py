@@ -214,25 +214,51 @@ class LayerWorkload:
         for p in range(len(self.projs)):
             self.h_y[p].copy_(self.y[p], non_blocking=True)
 
-    # ---- end-to-end arm, pipelined: a few lanes (own stream, device inputs, outputs, plan, workspace) take
-    # alternate steps, so the host <-> device copies of one step overlap the kernels of the other
-    E2E_BLOCK = 12  # steps issued per call of e2e_block (one CUDA graph holds that many)
-    E2E_LANES = 3
+    # ---- end-to-end arm, pipelined: one stream copies inputs in, one runs the kernels, one copies results out; a
+    # few buffer sets (device inputs, outputs, plan, workspace, pinned result buffers) rotate through them, so the
+    # host <-> device copies of a step run beside the kernels of its neighbours while the kernels of different
+    # steps never share the GPU
+    E2E_BLOCK = 48  # steps issued per call of e2e_block (one CUDA graph holds that many)
+    E2E_LANES = 3   # buffer sets
+
+    @staticmethod
+    def _packed(like, device, pin=False):
+        """One flat byte buffer holding tensors shaped like `like` at 256-byte offsets, and the views into it."""
+        offs, total = [], 0
+        for t in like:
+            offs.append(total)
+            total += (t.numel() * t.element_size() + 255) // 256 * 256
+        flat = torch.empty(total, dtype=torch.uint8, device=device)
+        if pin:
+            flat = flat.pin_memory()
+        views = [flat[o:o + t.numel() * t.element_size()].view(t.dtype).view(t.shape) for o, t in zip(offs, like)]
+        return flat, views
 
     def _make_lanes(self):
         moin, dev = self.moin, self.dev
         lanes = []
+        ins = [self.queries[0]] + [xs[0] for xs in self.x]
+        # a step's inputs (and its results) travel as ONE copy each way: host-side they sit packed in one pinned buffer
+        self.h_in = []
+        for j in range(self.n_host):
+            flat, views = self._packed(ins, "cpu", pin=True)
+            views[0].copy_(self.h_q[j])
+            for p in range(len(self.projs)):
+                views[1 + p].copy_(self.h_x[p][j])
+            self.h_in.append(flat)
         for k in range(self.E2E_LANES):
-            d_q = torch.empty_like(self.queries[0])
-            d_x = [torch.empty_like(xs[0]) for xs in self.x]
-            y = [torch.empty_like(t) for t in self.y]
+            d_in, in_views = self._packed(ins, dev)
+            d_out, y = self._packed(self.y, dev)
+            d_q, d_x = in_views[0], in_views[1:]
             lanes.append({
-                "stream": torch.cuda.Stream(), "d_q": d_q, "d_x": d_x, "y": y,
-                "h_y": [torch.empty_like(t, device="cpu").pin_memory() for t in self.y],
+                "d_q": d_q, "d_x": d_x, "y": y, "d_in": d_in, "d_out": d_out,
+                "h_out": torch.empty(d_out.numel(), dtype=torch.uint8).pin_memory(),
                 "req_expert": torch.empty(self.R, dtype=torch.int32, device=dev),
                 "plan": moin.Plan(self.T, self.E, dev, self.mode),
                 "ws": torch.empty_like(self.ws),
                 "groups": [moin.JobGroup([(d_x[p], self.W[p], self.pools[p], y[p]) for p in g]) for g in self.groups]})
+        self.e2e_streams = [torch.cuda.Stream() for _ in range(3)]   # copy in, kernels, copy out
+        self.h2d, self.d2h = lanes[0]["d_in"].numel(), lanes[0]["d_out"].numel()
         return lanes
 
     def e2e_block(self, b: int):
@@ -241,24 +267,40 @@ class LayerWorkload:
             self.lanes = self._make_lanes()
         moin = self.moin
         origin = torch.cuda.current_stream()
-        for lane in self.lanes:
-            lane["stream"].wait_stream(origin)
+        s_in, s_run, s_out = self.e2e_streams
+        for st in self.e2e_streams:
+            st.wait_stream(origin)
+        # per buffer set: events of its last use inside this block (the block's ends are full joins)
+        ran = [None] * self.E2E_LANES     # kernels done: the device inputs may be overwritten
+        out = [None] * self.E2E_LANES     # results copied out: the device outputs may be overwritten
         for k in range(self.E2E_BLOCK):
             step = b * self.E2E_BLOCK + k
-            i, lane = step % ROTATE, self.lanes[step % self.E2E_LANES]
+            n = step % self.E2E_LANES
+            i, lane = step % ROTATE, self.lanes[n]
             j = i % self.n_host
-            with torch.cuda.stream(lane["stream"]):
-                lane["d_q"].copy_(self.h_q[j], non_blocking=True)
-                for p in range(len(self.projs)):
-                    lane["d_x"][p].copy_(self.h_x[p][j], non_blocking=True)
+            with torch.cuda.stream(s_in):
+                if ran[n] is not None:
+                    s_in.wait_event(ran[n])
+                lane["d_in"].copy_(self.h_in[j], non_blocking=True)
+                ready = torch.cuda.Event()
+                ready.record(s_in)
+            with torch.cuda.stream(s_run):
+                s_run.wait_event(ready)
+                if out[n] is not None:
+                    s_run.wait_event(out[n])
                 moin.route(self.routers[i], lane["d_q"], out_expert=lane["req_expert"])
                 moin.plan_build(lane["req_expert"], self.E, self.mode, plan=lane["plan"])
                 for jg in lane["groups"]:
                     moin.lora_linear_group(lane["plan"], jg, self.scale, workspace=lane["ws"])
-                for p in range(len(self.projs)):
-                    lane["h_y"][p].copy_(lane["y"][p], non_blocking=True)
-        for lane in self.lanes:
-            origin.wait_stream(lane["stream"])
+                ran[n] = torch.cuda.Event()
+                ran[n].record(s_run)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ran[n])
+                lane["h_out"].copy_(lane["d_out"], non_blocking=True)
+                out[n] = torch.cuda.Event()
+                out[n].record(s_out)
+        for st in self.e2e_streams:
+            origin.wait_stream(st)
 
     def distinct(self) -> float:
         vals = []
@@ -875,11 +917,12 @@ def main():
     e2e_steps = max(5, args.steps // 4)
     e2e_mode = "one step after the other"
     if kind == "decode" and use_graph and wl.cache is None:
-        # pipelined: blocks of E2E_BLOCK steps on a few lanes, the copies of a step beside the kernels of its neighbour
+        # pipelined: blocks of E2E_BLOCK steps, the copies of a step beside the kernels of its neighbours
         blocks = max(2, e2e_steps // wl.E2E_BLOCK)
         ms_blk, _ = timed_loop(world, wl.e2e_block, blocks, 3, True)
         ms_e2e = ms_blk / wl.E2E_BLOCK
-        e2e_mode = f"{wl.E2E_LANES} lanes, CUDA graphs of {wl.E2E_BLOCK} steps"
+        e2e_mode = (f"copy-in / kernel / copy-out streams over {wl.E2E_LANES} buffer sets, one packed copy each way per step, "
+                    f"CUDA graphs of {wl.E2E_BLOCK} steps")
     else:
         ms_e2e, _ = timed_loop(world, wl.step_e2e, e2e_steps, max(3, args.warmup // 2), use_graph)
     ms_e2e = max_over_ranks(world, ms_e2e)

@@ -57,3 +57,34 @@ def test_decode_step_replayed_from_a_cuda_graph():
         err = np.linalg.norm(got - want) / np.linalg.norm(want)
         assert err <= REL_FRO, (name, err)
         assert (np.abs(got - want) <= ELEM_TOL * (1 + np.abs(want))).all(), name
+
+
+def test_end_to_end_arm_delivers_the_step_results_to_the_host():
+    """The pipelined end-to-end arm (packed pinned inputs -> copy-in stream -> kernels -> copy-out stream -> pinned
+    results, several buffer sets in flight, replayed from a CUDA graph) must leave in host memory exactly what the
+    plain step leaves on the device for the same batch."""
+    wl = bench.LayerWorkload("decode", str(DEV))
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        wl.e2e_block(0)                       # eager once (also builds the buffer sets)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            wl.e2e_block(0)
+        for lane in wl.lanes:
+            lane["h_out"].zero_()
+        g.replay()
+        stream.synchronize()
+    assert moin.device_status()["timeout_flag"] == 0
+    # the last use of buffer set n inside block 0 is step k = E2E_BLOCK - E2E_LANES + n ... E2E_BLOCK - 1
+    for k in range(wl.E2E_BLOCK - wl.E2E_LANES, wl.E2E_BLOCK):
+        n, i = k % wl.E2E_LANES, k % bench.ROTATE
+        wl.step(i)
+        torch.cuda.synchronize()
+        flat = wl.lanes[n]["h_out"]
+        off = 0
+        for p, y in enumerate(wl.y):
+            nbytes = y.numel() * 2
+            got = flat[off:off + nbytes].view(torch.bfloat16).view(y.shape)
+            assert torch.equal(got, y.cpu()), (k, wl.projs[p][0])
+            off += (nbytes + 255) // 256 * 256
