@@ -6,7 +6,8 @@
 //              multi-stage shared-memory ring, completion on mbarriers
 //   warp 1     allocates TMEM, issues tcgen05.mma (one thread), commits stage release and
 //              accumulator-ready barriers
-//   warps 2-5  epilogue: tcgen05.ld of the accumulator (TMEM lane = tile row), then one of
+//   warps 2-9  epilogue, two warps per TMEM lane quarter (half of the tile's columns each): tcgen05.ld of the
+//              accumulator (TMEM lane = tile row), then one of
 //              EPI_STORE   y = bf16(acc) (+ optional fp32 copy)
 //              EPI_ROUTER  running (max, argmax) of acc * inv_norm[col], merged across tiles with a
 //                          64-bit atomicMax on (orderable(sim) << 32 | ~col): order independent,
@@ -27,7 +28,7 @@
 namespace moin {
 
 constexpr int kBM = 128, kBK = 64;
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 320;
 enum { EPI_STORE = 0, EPI_ROUTER = 1, EPI_SHRINK = 2, EPI_ROUTER2 = 3 };   // ROUTER2: best and runner-up
 
 constexpr int kMaxShrinkJobs = 3;
@@ -93,8 +94,8 @@ template <int BN> struct TcCfg {
   static constexpr int kStageBytes = (kBM + BN) * kBK * 2;
   static constexpr int kStages = (200 * 1024) / kStageBytes > 8 ? 8 : (200 * 1024) / kStageBytes;
   static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;   // power of two for BN in {64,128,256}
-  // output staging of the store epilogue: per epilogue warp two [32 rows x 64 columns] bf16 buffers
-  static constexpr int kOutBytes = 4 * 2 * 32 * 128;
+  // output staging of the store epilogue: per epilogue warp one [32 rows x 64 columns] bf16 buffer
+  static constexpr int kOutBytes = 8 * 32 * 128;
   static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*align*/ + 1024 /*barriers*/ + kOutBytes;
 };
 
@@ -124,7 +125,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull0 + 8 * a, 1);
-      mbar_init(tempty0 + 8 * a, 128);
+      mbar_init(tempty0 + 8 * a, 256);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -244,11 +245,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
     const int q = warp & 3;             // TMEM lane quarter this warp may read
     const int trow = q * 32 + lane;     // row of the tile owned by this thread
     uint32_t lt = 0;
-    uint32_t n_st = 0;                  // tiled stores issued by this warp so far (two staging buffers in turn)
+    uint32_t n_st = 0;                  // tiled stores issued by this warp so far
+    const int wh = (warp - 2) >> 2;     // which half of the tile's columns this warp takes
+    const int c_lo = wh * (BN / 2), c_hi = c_lo + BN / 2;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++lt) {
       int row0, rows, n0, slot;
@@ -270,11 +273,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const bool staged = (EPI == EPI_STORE) && p.tma_store && (q * 32 + 32 <= rows);
       if (staged) {
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 64) {
+        for (int c = (BN >= 128 ? c_lo : 0); c < (BN >= 128 ? c_hi : (wh == 0 ? BN : 0)); c += 64) {
           if (n0 + c >= p.N) break;
-          const uint32_t buf = out0 + (uint32_t)q * 8192u + (n_st & 1u) * 4096u;
-          if (n_st >= 2) {               // the store that last read this buffer is the one before the newest
-            if (lane == 0) bulk_wait_read<1>();
+          const uint32_t buf = out0 + (uint32_t)(wh * 4 + q) * 4096u;
+          if (n_st >= 1) {               // the store that last read this buffer
+            if (lane == 0) bulk_wait_read<0>();
             __syncwarp();
           }
 #pragma unroll
@@ -302,7 +305,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
 #pragma unroll 1
-      for (int c = 0; c < ncols && !staged; c += 32) {
+      for (int c = c_lo; c < min(ncols, c_hi) && !staged; c += 32) {
         if (n0 + c >= p.N) break;
         uint32_t v[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c, v);
