@@ -28,7 +28,9 @@
 namespace moin {
 
 constexpr int kBM = 128, kBK = 64;
-constexpr int kTcThreads = 320;
+constexpr int kTcThreads = 320;      // producer warp, MMA warp, eight epilogue warps
+constexpr int kTcThreadsLean = 192;  // four epilogue warps and no output staging: the launch that runs beside the
+                                     // adapter streams at decode size and should leave them registers and shared memory
 enum { EPI_STORE = 0, EPI_ROUTER = 1, EPI_SHRINK = 2, EPI_ROUTER2 = 3 };   // ROUTER2: best and runner-up
 
 constexpr int kMaxShrinkJobs = 3;
@@ -125,7 +127,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull0 + 8 * a, 1);
-      mbar_init(tempty0 + 8 * a, 256);
+      mbar_init(tempty0 + 8 * a, blockDim.x - 64);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -250,8 +252,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int trow = q * 32 + lane;     // row of the tile owned by this thread
     uint32_t lt = 0;
     uint32_t n_st = 0;                  // tiled stores issued by this warp so far
-    const int wh = (warp - 2) >> 2;     // which half of the tile's columns this warp takes
-    const int c_lo = wh * (BN / 2), c_hi = c_lo + BN / 2;
+    // eight epilogue warps share a tile's columns in halves; a lean launch (kTcThreadsLean) has four, all columns each
+    const int wh = (warp - 2) >> 2;
+    const int c_w = (blockDim.x > kTcThreadsLean) ? BN / 2 : BN;
+    const int c_lo = wh * c_w, c_hi = c_lo + c_w;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++lt) {
       int row0, rows, n0, slot;
@@ -273,7 +277,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const bool staged = (EPI == EPI_STORE) && p.tma_store && (q * 32 + 32 <= rows);
       if (staged) {
 #pragma unroll 1
-        for (int c = (BN >= 128 ? c_lo : 0); c < (BN >= 128 ? c_hi : (wh == 0 ? BN : 0)); c += 64) {
+        for (int c = (c_w >= 64 ? c_lo : 0); c < (c_w >= 64 ? c_hi : (wh == 0 ? BN : 0)); c += 64) {
           if (n0 + c >= p.N) break;
           const uint32_t buf = out0 + (uint32_t)(wh * 4 + q) * 4096u;
           if (n_st >= 1) {               // the store that last read this buffer
@@ -452,15 +456,17 @@ moin_status make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t
 template <int BN, int EPI>
 static moin_status launch_cfg(HostState* hs, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& a2,
                               const CUtensorMap& a3, const CUtensorMap& b2, const TcParams& p, long max_tiles,
-                              cudaStream_t stream, const CUtensorMap* b3 = nullptr, const CUtensorMap* ymap = nullptr) {
+                              cudaStream_t stream, const CUtensorMap* b3 = nullptr, const CUtensorMap* ymap = nullptr,
+                              bool lean = false) {
   using Cfg = TcCfg<BN>;
   constexpr int slot = OPTIN_TC_GEMM + 4 * (BN == 256 ? 2 : BN == 128 ? 1 : 0) + EPI;
   cudaError_t e = ensure_smem_optin(slot, tc_gemm_kernel<BN, EPI>, Cfg::kSmemBytes);
   if (e != cudaSuccess) return record_cuda(e);
   long grid = max_tiles < hs->n_sms ? max_tiles : hs->n_sms;
   if (grid < 1) grid = 1;
-  tc_gemm_kernel<BN, EPI><<<(int)grid, kTcThreads, Cfg::kSmemBytes, stream>>>(a, b, a2, a3, b2, b3 ? *b3 : b2,
-                                                                               ymap ? *ymap : a, p);
+  const int threads = lean ? kTcThreadsLean : kTcThreads;
+  const size_t smem = lean ? Cfg::kSmemBytes - Cfg::kOutBytes : Cfg::kSmemBytes;   // (lean launches never stage)
+  tc_gemm_kernel<BN, EPI><<<(int)grid, threads, smem, stream>>>(a, b, a2, a3, b2, b3 ? *b3 : b2, ymap ? *ymap : a, p);
   return record_cuda(cudaGetLastError());
 }
 
@@ -517,9 +523,10 @@ moin_status launch_tc_gemm(HostState* hs, const __nv_bfloat16* x, const __nv_bfl
     p.tma_store = 1;
   }
   const long tiles = tiles_m * ((d_out + bn - 1) / bn);
-  if (bn == 256) return launch_cfg<256, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream, nullptr, &ym);
-  if (bn == 128) return launch_cfg<128, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream, nullptr, &ym);
-  return launch_cfg<64, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream, nullptr, &ym);
+  const bool lean = p.tma_store == 0;
+  if (bn == 256) return launch_cfg<256, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream, nullptr, &ym, lean);
+  if (bn == 128) return launch_cfg<128, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream, nullptr, &ym, lean);
+  return launch_cfg<64, EPI_STORE>(hs, a, b, a, a, b, p, tiles, stream, nullptr, &ym, lean);
 }
 
 moin_status launch_tc_router(HostState* hs, const __nv_bfloat16* q, const __nv_bfloat16* c, const float* inv_norm,
