@@ -53,7 +53,7 @@ struct TcParams {
   int ldy;
   float scale;                 // EPI_SHRINK
   // EPI_SHRINK over several projections that share the plan, K and the rank (n_jobs in 1..kMaxShrinkJobs):
-  // tile index = job * row tiles + row tile; job j reads x through the j-th A-side map and its pool through
+  // tile index = row tile * n_jobs + job; job j reads x through the j-th A-side map and its pool through
   // the j-th B-side map, looks its slot up in slot_tabs[j] and writes ys[j] / ys_lo[j].  n_jobs = 0: one job
   // described by slot_of_expert / y / y_lo.
   int n_jobs;
@@ -153,9 +153,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   auto tile_info = [&](int tile, int& row0, int& rows, int& n0, int& slot) {
     int tm = tile / tiles_n;
     n0 = (tile - tm * tiles_n) * BN;
-    if (EPI == EPI_SHRINK && n_jobs > 1) {
-      job = tm / tiles_m;
-      tm -= job * tiles_m;
+    if (EPI == EPI_SHRINK && n_jobs > 1) {   // the projections of one row tile side by side: its x tile is read once
+      job = tm % n_jobs;                     // from HBM and found in L2 by the CTAs next door
+      tm /= n_jobs;
     }
     slot = -1;
     if (planned) {
