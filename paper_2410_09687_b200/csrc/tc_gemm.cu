@@ -57,6 +57,10 @@ struct TcParams {
   // the j-th B-side map, looks its slot up in slot_tabs[j] and writes ys[j] / ys_lo[j].  n_jobs = 0: one job
   // described by slot_of_expert / y / y_lo.
   int n_jobs;
+  // ... or, when they also share x and their ranks fit one tile side by side (n_stack * stack_r <= BN): ONE pass
+  // over x, the adapters' rows stacked in the B operand (job j at rows j * stack_r), N = n_stack * stack_r
+  // accumulator columns, column group j stored to ys[j] / ys_lo[j].  n_stack > 1 implies n_jobs = 1.
+  int n_stack, stack_r;
   const int* slot_tabs[3];
   __nv_bfloat16* ys[3];
   __nv_bfloat16* ys_lo[3];
@@ -150,6 +154,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   int job = 0;   // projection of the current tile (EPI_SHRINK with several jobs), set by tile_info
   int r_use = (EPI == EPI_SHRINK) ? p.N : p.tail_r;   // rank of the current tile's adapter, set by tile_info
+  const bool stacked = (EPI == EPI_SHRINK) && p.n_stack > 1;
+  int st_slot[kMaxShrinkJobs] = {-1, -1, -1}, st_ruse[kMaxShrinkJobs] = {0, 0, 0};   // stacked: per projection
   auto tile_info = [&](int tile, int& row0, int& rows, int& n0, int& slot) {
     int tm = tile / tiles_n;
     n0 = (tile - tm * tiles_n) * BN;
@@ -165,7 +171,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int* tab = p.slot_of_expert;
       if (EPI == EPI_SHRINK && p.n_jobs > 0) tab = (job == 0) ? p.slot_tabs[0] : (job == 1) ? p.slot_tabs[1] : p.slot_tabs[2];
       if (e >= 0 && tab) slot = tab[e];
-      if (EPI == EPI_SHRINK || EPI == EPI_STORE) {
+      if (stacked) {
+#pragma unroll
+        for (int j = 0; j < kMaxShrinkJobs; ++j) {
+          st_slot[j] = (j < p.n_stack && e >= 0) ? p.slot_tabs[j][e] : -1;
+          st_ruse[j] = (st_slot[j] >= 0 && p.rank_tabs[j]) ? min(p.rank_tabs[j][st_slot[j]], p.stack_r) : p.stack_r;
+        }
+        slot = st_slot[0];
+      } else if (EPI == EPI_SHRINK || EPI == EPI_STORE) {
         const int r_full = (EPI == EPI_SHRINK) ? p.N : p.tail_r;
         const int* rt = (EPI == EPI_STORE) ? p.slot_rank
                                            : (job == 0 ? p.rank_tabs[0] : job == 1 ? p.rank_tabs[1] : p.rank_tabs[2]);
@@ -193,9 +206,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t s = it % S, ph = (it / S) & 1u;
           if (!(ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag, p.status, 1))) break;
           const uint32_t sa = tiles_base + s * Cfg::kStageBytes, sb = sa + kBM * kBK * 2;
-          const uint32_t b_rows = (kb < nkb_main && p.b_box_rows > 0) ? (uint32_t)p.b_box_rows : (uint32_t)BN;
+          const uint32_t b_rows = stacked ? (uint32_t)(p.n_stack * p.stack_r)
+                                          : (kb < nkb_main && p.b_box_rows > 0) ? (uint32_t)p.b_box_rows : (uint32_t)BN;
           mbar_expect_tx(full0 + 8 * s, (kBM + b_rows) * kBK * 2);
-          if (kb < nkb_main) {
+          if (stacked) {
+            tma_load_2d(sa, &tmA, full0 + 8 * s, kb * kBK, row0);
+#pragma unroll
+            for (int j = 0; j < kMaxShrinkJobs; ++j)
+              if (j < p.n_stack)   // (a projection without this adapter loads slot 0: its columns are not stored)
+                tma_load_2d(sb + (uint32_t)(j * p.stack_r) * kBK * 2, j == 0 ? &tmB : j == 1 ? &tmB2 : &tmB3, full0 + 8 * s,
+                            kb * kBK, (st_slot[j] >= 0 ? st_slot[j] : 0) * p.stack_r);
+          } else if (kb < nkb_main) {
             const CUtensorMap* ma = &tmA;
             const CUtensorMap* mb = &tmB;
             if (EPI == EPI_SHRINK && job > 0) {
@@ -334,7 +355,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               }
             }
           }
-        } else if (row_ok && (EPI == EPI_STORE || slot >= 0)) {
+        } else if (row_ok && (EPI == EPI_STORE || stacked || slot >= 0)) {
           const float sc = (EPI == EPI_SHRINK) ? p.scale : 1.f;
           __nv_bfloat16* ybase = p.y;
           __nv_bfloat16* ylo_base = p.y_lo;
@@ -342,17 +363,28 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             ybase = (job == 0) ? p.ys[0] : (job == 1) ? p.ys[1] : p.ys[2];
             ylo_base = (job == 0) ? p.ys_lo[0] : (job == 1) ? p.ys_lo[1] : p.ys_lo[2];
           }
-          __nv_bfloat16* yrow = ybase + grow * (size_t)p.ldy + n0 + c;
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
-            if (n0 + c + j < p.N) {  // N is a multiple of 8
+            int cj = n0 + c + j;     // first of eight columns (N is a multiple of 8); stacked: of its projection
+            int ru = r_use;
+            bool keep = cj < p.N;
+            if (stacked && keep) {
+              const int jb = cj / p.stack_r;
+              cj -= jb * p.stack_r;
+              keep = (jb == 0 ? st_slot[0] : jb == 1 ? st_slot[1] : st_slot[2]) >= 0;
+              ru = jb == 0 ? st_ruse[0] : jb == 1 ? st_ruse[1] : st_ruse[2];
+              ybase = jb == 0 ? p.ys[0] : jb == 1 ? p.ys[1] : p.ys[2];
+              ylo_base = jb == 0 ? p.ys_lo[0] : jb == 1 ? p.ys_lo[1] : p.ys_lo[2];
+            }
+            __nv_bfloat16* yrow = ybase + grow * (size_t)p.ldy + cj - j;
+            if (keep) {
               float f[8];
 #pragma unroll
               for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]) * sc;
               if (EPI == EPI_SHRINK) {   // function between the low-rank matrices; nothing beyond the adapter's rank
 #pragma unroll
                 for (int e = 0; e < 8; ++e)
-                  f[e] = (n0 + c + j + e < r_use) ? lora_act(__uint_as_float(v[j + e]), p.act) * sc : 0.f;
+                  f[e] = (cj + e < ru) ? lora_act(__uint_as_float(v[j + e]), p.act) * sc : 0.f;
               }
               uint4 o;
               o.x = pack_bf16(f[0], f[1]);
@@ -366,10 +398,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 l.y = pack_bf16(f[2] - bf16_lo(o.y), f[3] - bf16_hi(o.y));
                 l.z = pack_bf16(f[4] - bf16_lo(o.z), f[5] - bf16_hi(o.z));
                 l.w = pack_bf16(f[6] - bf16_lo(o.w), f[7] - bf16_hi(o.w));
-                *reinterpret_cast<uint4*>(ylo_base + grow * (size_t)p.ldy + n0 + c + j) = l;
+                *reinterpret_cast<uint4*>(ylo_base + grow * (size_t)p.ldy + cj) = l;
               }
               if (EPI == EPI_STORE && p.y0) {
-                float* y0row = p.y0 + grow * (size_t)p.ldy + n0 + c + j;
+                float* y0row = p.y0 + grow * (size_t)p.ldy + cj;
                 *reinterpret_cast<uint4*>(y0row) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                 *reinterpret_cast<uint4*>(y0row + 4) = make_uint4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
               }
@@ -580,6 +612,21 @@ moin_status launch_tc_shrink_group(HostState* hs, const PlanView& pv, const moin
     bA[j] = bA[0];
   }
   ProfScope prof(MOIN_K_SHRINK_TC, 1, stream);
+  // Projections that read the same x and whose ranks fit one tile side by side take ONE pass over x: their
+  // adapters' rows are stacked in the B operand and the accumulator's column groups go to their own outputs.
+  bool same_x = n_jobs > 1 && n_jobs * r <= 256;
+  for (int j = 1; j < n_jobs; ++j) same_x = same_x && xs[j] == xs[0];
+  if (same_x) {
+    p.n_jobs = 1;
+    p.n_stack = n_jobs;
+    p.stack_r = r;
+    p.N = n_jobs * r;
+    p.b_box_rows = 0;
+    const int nt = n_jobs * r;
+    if (nt > 128) return launch_cfg<256, EPI_SHRINK>(hs, ax[0], bA[0], ax[1], ax[2], bA[1], p, (long)T, stream, &bA[2]);
+    if (nt > 64) return launch_cfg<128, EPI_SHRINK>(hs, ax[0], bA[0], ax[1], ax[2], bA[1], p, (long)T, stream, &bA[2]);
+    return launch_cfg<64, EPI_SHRINK>(hs, ax[0], bA[0], ax[1], ax[2], bA[1], p, (long)T, stream, &bA[2]);
+  }
   // upper bound on row tiles without reading the plan back: every run adds at most one partial tile;
   // the grid is capped at the SM count and the kernel reads the true count
   if (r > 64) return launch_cfg<128, EPI_SHRINK>(hs, ax[0], bA[0], ax[1], ax[2], bA[1], p, (long)T * n_jobs, stream, &bA[2]);

@@ -163,6 +163,39 @@ def test_grouped_projections_equal_single_calls(mode):
         assert_layer_close(y, oracle_layer(case), case.name)
 
 
+@pytest.mark.parametrize("r,n_proj", [(16, 3), (32, 3), (64, 2), (64, 3), (128, 2)])
+def test_grouped_projections_that_share_their_input(r, n_proj):
+    """{q, k, v} / {gate, up}-like groups over long runs: the projections read the SAME x, so their shrinks are one
+    pass over it with the adapters' rows side by side in one tile (where n_proj * r fits: up to 256).  Every pool
+    misses a different expert and gives its slots different ranks; each output must be bit-identical to the
+    single call and match the oracle."""
+    rng = mi.np_rng(29, r)
+    E, T, d_in = 12, 300, 256
+    te = np.repeat(rng.integers(0, E, size=4), [130, 70, 37, 63]).astype(np.int32)
+    te[5:9] = -1
+    plan = moin.plan_build(torch.from_numpy(te).to(DEV), E, moin.PLAN_TILES)
+    x = mi.normal_bf16((T, d_in), 1.0, 29, r, 1).to(DEV)
+    jobs, refs, singles = [], [], []
+    for i in range(n_proj):
+        d_out = [256, 64, 136][i]
+        pool = mi.make_pool(E, r, d_in, d_out, 29, 10 + i, missing=(int(te[0]) if i == 1 else (i + 2) % E,))
+        n_slots = pool.A.shape[0]
+        ranks = np.array([[r, 8, r // 2, 0][(s_ + i) % 4] for s_ in range(n_slots)], np.int32)
+        W = mi.normal_bf16((d_out, d_in), 0.05, 29, r, 20 + i)
+        gp = moin.Pool(pool.A.to(DEV), pool.B.to(DEV), pool.slot_of_expert.to(DEV), slot_rank=torch.from_numpy(ranks).to(DEV))
+        y = torch.empty(T, d_out, dtype=torch.bfloat16, device=DEV)
+        jobs.append((x, W.to(DEV), gp, y))
+        singles.append(moin.lora_linear(plan, x, W.to(DEV), gp, 2.0).clone())
+        refs.append(oracle.lora_linear(mi.bf16_bits(x.cpu()), mi.bf16_bits(W), mi.bf16_bits(pool.A), mi.bf16_bits(pool.B), te,
+                                       pool.slot_of_expert.numpy(), 2.0, slot_rank=ranks))
+    moin.lora_linear_group(plan, moin.JobGroup(jobs), 2.0)
+    torch.cuda.synchronize()
+    assert moin.device_status()["timeout_flag"] == 0
+    for i, ((_, _, _, y), y1, ref) in enumerate(zip(jobs, singles, refs)):
+        assert torch.equal(y, y1), i
+        assert_layer_close(y, ref, f"shared input, projection {i}")
+
+
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_seeded_random_shapes_in_every_plan_mode(seed):
     # ranks, widths (also not multiples of 16 / 64), segment structures (runs, interleaved tokens, base-only
